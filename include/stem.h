@@ -1,0 +1,154 @@
+/*
+ * stem.h - C ABI of the Stem sparse causal prefill attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the hot path of Algorithm 1 of "Stem" (arxiv 2603.06274):
+ *
+ *   stem_score           Alg. 1 step 1 (block pooling of Q and K, max-pooled value magnitude)
+ *                        and step 3a (Output-Aware Metric, Eq. 7) on pooled blocks
+ *   stem_select          Alg. 1 steps 3b-3c: Token Position-Decay budget (Eq. 3, block units)
+ *                        and per-row top-k with the forced stem / local blocks
+ *   stem_sparse_prefill  Alg. 1 step 3d: exact causal softmax attention over the listed blocks
+ *   stem_prefill         all of Algorithm 1 on one stream, no host synchronisation
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned.
+ *     Q, K, V, O hold bf16.  Element (t, h, c) of Q is at Q[t*q_stride_tok + h*q_stride_head + c]
+ *     (strides in elements, c contiguous, 0 <= c < head_dim = 128); K and V share
+ *     kv_stride_tok / kv_stride_head.  O is contiguous [T, num_q_heads, head_dim].
+ *     Sequences are packed along t (varlen): sequence b owns tokens
+ *     cu_seqlens[b] .. cu_seqlens[b+1]-1 and never attends to another sequence.
+ *   - Query-block rows are numbered globally, sequence-major: R = row_offset(b) + r,
+ *     r = 0 .. N_blk(b)-1, N_blk(b) = ceil(len_b / block); R_tot = sum_b N_blk(b).
+ *   - Index lists: sel_idx is int32 [num_q_heads, R_tot, k_max], sel_cnt int32
+ *     [num_q_heads, R_tot].  Row (h, R) holds sel_cnt valid block ids, local to the
+ *     sequence, strictly ascending, each <= r; the remaining entries are -1.
+ *   - `stream` is a cudaStream_t passed as void*.  Hot calls enqueue work on it and return;
+ *     they never allocate, never synchronise and never throw.
+ *   - Return value: STEM_OK (0) or a negative stem_status.  Nothing is enqueued when a call
+ *     returns STEM_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE.
+ *   - Device-side waits are bounded; a wait that gives up records a code in the workspace,
+ *     the kernel returns early, and stem_check_status reports STEM_ERR_DEVICE_TIMEOUT.
+ */
+#ifndef STEM_H_
+#define STEM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  STEM_OK = 0,
+  STEM_ERR_INVALID_ARG = -1,    /* null pointer, bad size, misaligned pointer or stride           */
+  STEM_ERR_UNSUPPORTED = -2,    /* head_dim != 128, block not in {64,128}, heads not divisible, ... */
+  STEM_ERR_WORKSPACE = -3,      /* workspace missing or smaller than stem_plan_query reports      */
+  STEM_ERR_CUDA = -4,           /* a CUDA runtime / driver call or a kernel launch failed         */
+  STEM_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait gave up (see stem_check_status)     */
+} stem_status;
+
+/* Problem statement of Algorithm 1 (inputs Q, K, V; hyper-parameters k_start, mu, B, beta) plus
+ * the forced-block settings of the paper's implementation details (4 initial + 4 local blocks,
+ * minimum total budget). Plain data; copied by stem_plan_create. */
+typedef struct {
+  int32_t batch;                  /* number of packed sequences, >= 1                              */
+  const int32_t* cu_seqlens_host; /* HOST pointer, [batch+1] token offsets, cu[0] = 0, increasing  */
+  int32_t num_q_heads;            /* H_q                                                           */
+  int32_t num_kv_heads;           /* H_kv, divides H_q; query head h reads kv head h / (H_q/H_kv)  */
+  int32_t head_dim;               /* must be 128                                                   */
+  int32_t block;                  /* B: 64 or 128                                                  */
+  int32_t budget_permille;        /* k_start = floor(budget_permille * N_blk / 1000) blocks        */
+  int32_t k_start_blocks;         /* if > 0, overrides budget_permille                             */
+  int32_t mu_num, mu_den;         /* decay ratio mu = mu_num/mu_den in (0,1]; 7/10 in the paper    */
+  int32_t stem_blocks;            /* initial blocks always kept (paper: 4), >= 0                   */
+  int32_t local_blocks;           /* trailing blocks always kept, diagonal included (paper: 4), >= 1 */
+  int32_t min_blocks;             /* lower bound of the per-row budget (paper: 54), >= 0           */
+  float beta;                     /* weight of the magnitude term of Eq. 7 (paper: 0.2)            */
+  float score_scale;              /* multiplies Qbar.Kbar in the metric; 0 means 1.0 (Eq. 7)       */
+  float softmax_scale;            /* 0 means 1/sqrt(head_dim) (Alg. 1 step d)                      */
+  int64_t q_stride_tok, q_stride_head;   /* elements; multiples of 8                               */
+  int64_t kv_stride_tok, kv_stride_head; /* elements; multiples of 8                               */
+} stem_config;
+
+typedef struct stem_plan stem_plan; /* opaque; owns small host and device tables only */
+
+/* Sizes a caller needs to allocate buffers for a plan. */
+typedef struct {
+  size_t workspace_bytes;       /* scratch the hot calls need (pooled tensors, lists, status)      */
+  int32_t total_tokens;         /* T                                                               */
+  int32_t total_q_blocks;       /* R_tot                                                           */
+  int32_t k_max;                /* longest index list = max_r k_eff(r)                             */
+  int64_t metric_elems;         /* per head: sum_b N_blk(b)^2, the size of one head of M           */
+  int64_t selected_blocks;      /* sum over heads and rows of the list lengths (exact)             */
+  int64_t causal_blocks;        /* sum over heads and rows of r+1 (admissible blocks)              */
+  int64_t selected_pairs;       /* unmasked (query, key) pairs inside the selected blocks          */
+  int64_t causal_pairs;         /* unmasked (query, key) pairs of dense causal attention           */
+} stem_plan_info;
+
+/* Builds the per-row budget table k_eff(r) (Eq. 3 in block units, i = r+1, clamped by the forced
+ * blocks, min_blocks and the r+1 causal blocks), the row maps and the work order of the attention
+ * kernel, and uploads them to the current CUDA device (the only allocation the library makes).
+ * Host work only plus one synchronous copy; call it outside the hot path. */
+int stem_plan_create(const stem_config* cfg, stem_plan** out_plan);
+int stem_plan_destroy(stem_plan* plan);
+int stem_plan_query(const stem_plan* plan, stem_plan_info* info);
+
+/* Copies the per-row budget table k_eff (int32 [R_tot], host memory) out of the plan. */
+int stem_plan_budget(const stem_plan* plan, int32_t* k_eff_host);
+
+/* Host-only form of the budget schedule (Eq. 3 in block units with the forced-block and
+ * min_blocks clamps): validates cfg and writes k_eff for every global row into k_eff_host
+ * (capacity entries; pass NULL to only count).  *r_tot receives R_tot.  Needs no CUDA device. */
+int stem_budget_table(const stem_config* cfg, int32_t* k_eff_host, int64_t capacity, int32_t* r_tot);
+
+/* Alg. 1 step 1 and step 3a.
+ *   Pools Q and K (block means over the valid tokens of each block) and V
+ *   (MV = max(0, max_t ln ||V_t||_2) per block) into the workspace, then, if M != NULL, writes
+ *   the Output-Aware Metric of Eq. 7 on pooled blocks,
+ *     M[h, m_off(b) + r*N_blk(b) + j] = score_scale * Qbar[h,r].Kbar[kv(h),j] + beta * MV[kv(h),j],
+ *   for causal blocks j <= r only (entries with j > r are not written).  M is fp32
+ *   [num_q_heads, metric_elems].  With M == NULL only the pooled tensors are produced. */
+int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* workspace,
+               size_t workspace_bytes, void* stream);
+
+/* Alg. 1 steps 3b-3c.
+ *   For every (head, row): keeps the forced blocks {0..stem-1} and {r-local+1..r}, then adds the
+ *   causal blocks of largest metric until the row holds k_eff(r) blocks.  Order: metric
+ *   descending, block id ascending on equal metric, -0 == +0, NaN below every number.
+ *   Reads M (layout above) if M != NULL, else recomputes metric rows from the pooled tensors a
+ *   preceding stem_score left in the same workspace.  Writes sel_idx / sel_cnt. */
+int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t* sel_cnt, void* workspace,
+                size_t workspace_bytes, void* stream);
+
+/* Alg. 1 step 3d.
+ *   O[t,h,:] = softmax_k( Q[t,h].K[k,kv(h)] * softmax_scale ) V over the keys k of the listed
+ *   blocks of t's row with position <= t.  sel_idx == NULL (with sel_cnt == NULL) means every
+ *   causal block, i.e. dense causal attention.  Lists must be ascending and within [0, r];
+ *   out-of-range ids are clamped, never dereferenced.  lse (fp32 [num_q_heads, T], natural-log
+ *   sum-exp of the scaled scores) is optional (NULL to skip). */
+int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, const int32_t* sel_idx,
+                        const int32_t* sel_cnt, void* O, float* lse, void* workspace, size_t workspace_bytes,
+                        void* stream);
+
+/* All of Algorithm 1: stem_score (without materialising M) -> stem_select -> stem_sparse_prefill on
+ * `stream`.  sel_idx / sel_cnt are optional outputs (both NULL: lists stay in the workspace). */
+int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
+                 int32_t* sel_cnt, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream`, then reads and clears the device status words of `workspace`.
+ * Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in a kernel gave up; outputs of that
+ * call are undefined) or STEM_ERR_CUDA.  detail (optional, HOST int32[4]) receives the raw words:
+ * {code, block index, role, barrier id}. */
+int stem_check_status(const stem_plan* plan, void* workspace, void* stream, int32_t* detail_host);
+
+/* Number of kernels the last hot call on this plan launched (for launch accounting). */
+int stem_last_launch_count(const stem_plan* plan);
+
+const char* stem_status_string(int status);
+int stem_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STEM_H_ */

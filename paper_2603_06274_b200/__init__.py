@@ -1,0 +1,11 @@
+"""Stem sparse causal prefill attention for NVIDIA B200 (sm_100a).
+
+The product is the C-ABI library ``libstem.so`` (see ``include/stem.h``); this package holds its
+CUDA sources, the in-tree build, a thin ctypes binding with the same entry-point names, and the
+seeded synthetic workloads used by the tests and the benchmark.
+"""
+from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    StemConfig, StemError, StemPlan, StemPlanInfo, load, library_path, status_string,
+    stem_check_status, stem_prefill, stem_score, stem_select, stem_sparse_prefill,
+)

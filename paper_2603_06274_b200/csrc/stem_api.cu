@@ -1,0 +1,398 @@
+// C ABI of libstem: argument checks, the plan (budget schedule, row maps, work orders) and the
+// stage sequencing.  All arithmetic of the method on tensors happens in the kernels; the only
+// method arithmetic here is the integer budget schedule of Eq. 3.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "stem_internal.h"
+
+namespace stem {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Token Position-Decay budget in block units (Eq. 3 with N -> N_blk, i = 1-indexed block row):
+//   k_blk(i) = floor(k_s - k_s (1 - mu) i / N_blk), then clamped from below by the forced blocks
+//   (stem + local, counted once where they overlap) and min_blocks, and from above by the i
+//   causal blocks.  Exact integer arithmetic.
+static int32_t budget_row(int64_t i, int64_t n_blk, int64_t k_s, const stem_config& c) {
+  const int64_t den = (int64_t)c.mu_den * n_blk;
+  const int64_t num = k_s * ((int64_t)c.mu_den * n_blk - (int64_t)(c.mu_den - c.mu_num) * i);
+  int64_t k = num / den;
+  const int64_t n_stem = std::min<int64_t>(c.stem_blocks, i);
+  const int64_t lo_local = std::max<int64_t>(0, i - c.local_blocks);
+  int64_t forced = n_stem + (i - lo_local) - std::max<int64_t>(0, n_stem - lo_local);
+  k = std::max<int64_t>(k, c.min_blocks);
+  k = std::max<int64_t>(k, forced);
+  k = std::min<int64_t>(k, i);
+  return (int32_t)k;
+}
+
+static int validate(const stem_config* c) {
+  if (!c || !c->cu_seqlens_host) return STEM_ERR_INVALID_ARG;
+  if (c->batch < 1 || c->num_q_heads < 1 || c->num_kv_heads < 1) return STEM_ERR_INVALID_ARG;
+  if (c->head_dim != kHeadDim) return STEM_ERR_UNSUPPORTED;
+  if (c->block != 64 && c->block != 128) return STEM_ERR_UNSUPPORTED;
+  if (c->num_q_heads % c->num_kv_heads != 0) return STEM_ERR_UNSUPPORTED;
+  if (c->num_q_heads / c->num_kv_heads > 32) return STEM_ERR_UNSUPPORTED;
+  if (c->mu_den <= 0 || c->mu_num <= 0 || c->mu_num > c->mu_den) return STEM_ERR_INVALID_ARG;
+  if (c->stem_blocks < 0 || c->local_blocks < 1 || c->min_blocks < 0) return STEM_ERR_INVALID_ARG;
+  if (c->k_start_blocks < 0 || c->budget_permille < 0 || c->budget_permille > 1000) return STEM_ERR_INVALID_ARG;
+  if (c->k_start_blocks == 0 && c->budget_permille == 0 && c->min_blocks == 0 && c->stem_blocks + c->local_blocks == 0)
+    return STEM_ERR_INVALID_ARG;
+  if (!(c->beta == c->beta) || !(c->score_scale == c->score_scale) || !(c->softmax_scale == c->softmax_scale))
+    return STEM_ERR_INVALID_ARG;
+  if (c->q_stride_tok % 8 || c->q_stride_head % 8 || c->kv_stride_tok % 8 || c->kv_stride_head % 8)
+    return STEM_ERR_INVALID_ARG;
+  if (c->q_stride_head < kHeadDim || c->kv_stride_head < kHeadDim) return STEM_ERR_INVALID_ARG;
+  if (c->q_stride_tok < kHeadDim || c->kv_stride_tok < kHeadDim) return STEM_ERR_INVALID_ARG;
+  if (c->cu_seqlens_host[0] != 0) return STEM_ERR_INVALID_ARG;
+  for (int b = 0; b < c->batch; ++b)
+    if (c->cu_seqlens_host[b + 1] <= c->cu_seqlens_host[b]) return STEM_ERR_INVALID_ARG;
+  return STEM_OK;
+}
+
+template <class T>
+static size_t push(std::vector<uint8_t>& blob, const std::vector<T>& v) {
+  size_t off = align_up(blob.size(), 256);
+  blob.resize(off + std::max<size_t>(v.size() * sizeof(T), 1));
+  if (!v.empty()) std::memcpy(blob.data() + off, v.data(), v.size() * sizeof(T));
+  return off;
+}
+
+}  // namespace stem
+
+using namespace stem;
+
+extern "C" {
+
+struct stem_plan {
+  Plan p;
+};
+
+int stem_version(void) { return 100; }
+
+const char* stem_status_string(int s) {
+  switch (s) {
+    case STEM_OK: return "ok";
+    case STEM_ERR_INVALID_ARG: return "invalid argument";
+    case STEM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case STEM_ERR_WORKSPACE: return "workspace missing or too small";
+    case STEM_ERR_CUDA: return "CUDA error";
+    case STEM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown status";
+  }
+}
+
+int stem_plan_create(const stem_config* cfg, stem_plan** out) {
+  if (!out) return STEM_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate(cfg);
+  if (rc != STEM_OK) return rc;
+
+  stem_plan* sp = new (std::nothrow) stem_plan();
+  if (!sp) return STEM_ERR_CUDA;
+  Plan& p = sp->p;
+  p.cfg = *cfg;
+  p.cu.assign(cfg->cu_seqlens_host, cfg->cu_seqlens_host + cfg->batch + 1);
+  p.cfg.cu_seqlens_host = nullptr;
+  p.score_scale = cfg->score_scale == 0.f ? 1.f : cfg->score_scale;
+  p.softmax_scale = cfg->softmax_scale == 0.f ? 1.f / std::sqrt((float)kHeadDim) : cfg->softmax_scale;
+
+  const int B = cfg->block, batch = cfg->batch, Hq = cfg->num_q_heads, Hkv = cfg->num_kv_heads;
+  const int g = Hq / Hkv;
+  p.T = p.cu[batch];
+
+  std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_len(batch), seq_nblk(batch),
+      seq_row_off(batch);
+  std::vector<int64_t> seq_m_off(batch);
+  int64_t m_off = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int32_t n = p.cu[b + 1] - p.cu[b];
+    const int32_t nb = (n + B - 1) / B;
+    seq_tok0[b] = p.cu[b];
+    seq_len[b] = n;
+    seq_nblk[b] = nb;
+    seq_row_off[b] = (int32_t)row_seq.size();
+    seq_m_off[b] = m_off;
+    m_off += (int64_t)nb * nb;
+    p.max_nblk = std::max(p.max_nblk, nb);
+    const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb) / 1000;
+    for (int32_t r = 0; r < nb; ++r) {
+      row_seq.push_back(b);
+      row_r.push_back(r);
+      row_tok0.push_back(p.cu[b] + r * B);
+      const int32_t ntok = std::min(B, n - r * B);
+      row_ntok.push_back(ntok);
+      const int32_t ke = budget_row(r + 1, nb, k_s, *cfg);
+      p.k_eff.push_back(ke);
+      p.k_max = std::max(p.k_max, ke);
+      const int64_t diag = (int64_t)ntok * (ntok + 1) / 2;
+      p.selected_blocks += ke;
+      p.causal_blocks += r + 1;
+      p.selected_pairs += (int64_t)(ke - 1) * ntok * B + diag;
+      p.causal_pairs += (int64_t)r * ntok * B + diag;
+    }
+  }
+  p.R_tot = (int32_t)row_seq.size();
+  p.m_tot = m_off;
+  p.selected_blocks *= Hq;
+  p.causal_blocks *= Hq;
+  p.selected_pairs *= Hq;
+  p.causal_pairs *= Hq;
+
+  // Score/select tiles: one CTA scores the g heads of a kv group for a run of consecutive rows.
+  // A tile holds at most 32 pooled query vectors and one fp32 metric row per vector in shared
+  // memory, which bounds the number of blocks per sequence.
+  const size_t ncols_pad = (size_t)(p.max_nblk + 63) / 64 * 64;
+  const size_t metric_smem_cap = 136 * 1024;  // what is left of 227 KB after the staging buffers
+  int nq_cap = 32;
+  while (nq_cap > g && (size_t)((nq_cap + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) nq_cap /= 2;
+  if ((size_t)((std::max(1, nq_cap / g) * g + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) {
+    delete sp;
+    return STEM_ERR_UNSUPPORTED;
+  }
+  p.sel_rows_per_tile = std::max(1, nq_cap / g);
+  p.sel_nq = p.sel_rows_per_tile * g;
+  std::vector<int32_t> tiles;
+  {
+    std::vector<std::pair<int32_t, std::pair<int32_t, int32_t>>> t;  // (last row, (seq, r0)), long rows first
+    for (int b = 0; b < batch; ++b)
+      for (int32_t r0 = 0; r0 < seq_nblk[b]; r0 += p.sel_rows_per_tile) t.push_back({r0, {b, r0}});
+    std::stable_sort(t.begin(), t.end(), [](auto& a, auto& b) { return a.first > b.first; });
+    for (auto& e : t) {
+      tiles.push_back(e.second.first);
+      tiles.push_back(e.second.second);
+    }
+    p.n_sel_tiles = (int32_t)t.size();
+  }
+
+  // Attention work order: kv-head-major so that the K/V of one kv head stay hot in L2; inside a
+  // kv head, rows by descending list length (longest first), the g heads of a row together.
+  std::vector<int32_t> work_sparse, work_dense;
+  {
+    std::vector<int32_t> by_len(p.R_tot), by_r(p.R_tot);
+    std::iota(by_len.begin(), by_len.end(), 0);
+    std::iota(by_r.begin(), by_r.end(), 0);
+    std::stable_sort(by_len.begin(), by_len.end(), [&](int a, int b) { return p.k_eff[a] > p.k_eff[b]; });
+    std::stable_sort(by_r.begin(), by_r.end(), [&](int a, int b) { return row_r[a] > row_r[b]; });
+    for (int kvh = 0; kvh < Hkv; ++kvh) {
+      for (int32_t R : by_len)
+        for (int q = 0; q < g; ++q) { work_sparse.push_back(kvh * g + q); work_sparse.push_back(R); }
+      for (int32_t R : by_r)
+        for (int q = 0; q < g; ++q) { work_dense.push_back(kvh * g + q); work_dense.push_back(R); }
+    }
+    p.n_items = p.R_tot * Hq;
+  }
+
+  // Workspace layout.
+  {
+    size_t off = 0;
+    p.ws.status = off; off = align_up(off + kStatusWords * 4, 256);
+    p.ws.qbar = off;   off = align_up(off + (size_t)Hq * p.R_tot * kHeadDim * 4, 256);
+    p.ws.kbar = off;   off = align_up(off + (size_t)Hkv * p.R_tot * kHeadDim * 4, 256);
+    p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
+    p.ws.sel_idx = off; off = align_up(off + (size_t)Hq * p.R_tot * p.k_max * 4, 256);
+    p.ws.sel_cnt = off; off = align_up(off + (size_t)Hq * p.R_tot * 4, 256);
+    p.ws.total = off;
+  }
+
+  // Upload tables.
+  if (cudaGetDevice(&p.device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&p.sm_count, cudaDevAttrMultiProcessorCount, p.device) != cudaSuccess) {
+    cudaGetLastError();
+    delete sp;
+    return STEM_ERR_CUDA;
+  }
+  std::vector<uint8_t> blob;
+  const size_t o_row_seq = push(blob, row_seq), o_row_r = push(blob, row_r), o_row_tok0 = push(blob, row_tok0),
+               o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
+               o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
+               o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off),
+               o_tiles = push(blob, tiles), o_ws = push(blob, work_sparse), o_wd = push(blob, work_dense);
+  if (cudaMalloc(&p.d_blob, blob.size()) != cudaSuccess ||
+      cudaMemcpy(p.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    if (p.d_blob) cudaFree(p.d_blob);
+    delete sp;
+    return STEM_ERR_CUDA;
+  }
+  const uint8_t* d = (const uint8_t*)p.d_blob;
+  p.rows.row_seq = (const int32_t*)(d + o_row_seq);
+  p.rows.row_r = (const int32_t*)(d + o_row_r);
+  p.rows.row_tok0 = (const int32_t*)(d + o_row_tok0);
+  p.rows.row_ntok = (const int32_t*)(d + o_row_ntok);
+  p.rows.row_keff = (const int32_t*)(d + o_keff);
+  p.rows.seq_tok0 = (const int32_t*)(d + o_seq_tok0);
+  p.rows.seq_len = (const int32_t*)(d + o_seq_len);
+  p.rows.seq_nblk = (const int32_t*)(d + o_seq_nblk);
+  p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
+  p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
+  p.d_sel_tiles = (const int32_t*)(d + o_tiles);
+  p.d_work_sparse = (const int32_t*)(d + o_ws);
+  p.d_work_dense = (const int32_t*)(d + o_wd);
+  *out = sp;
+  return STEM_OK;
+}
+
+int stem_plan_destroy(stem_plan* plan) {
+  if (!plan) return STEM_ERR_INVALID_ARG;
+  if (plan->p.d_blob) cudaFree(plan->p.d_blob);
+  delete plan;
+  return STEM_OK;
+}
+
+int stem_plan_query(const stem_plan* plan, stem_plan_info* info) {
+  if (!plan || !info) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  info->workspace_bytes = p.ws.total;
+  info->total_tokens = p.T;
+  info->total_q_blocks = p.R_tot;
+  info->k_max = p.k_max;
+  info->metric_elems = p.m_tot;
+  info->selected_blocks = p.selected_blocks;
+  info->causal_blocks = p.causal_blocks;
+  info->selected_pairs = p.selected_pairs;
+  info->causal_pairs = p.causal_pairs;
+  return STEM_OK;
+}
+
+int stem_plan_budget(const stem_plan* plan, int32_t* k_eff_host) {
+  if (!plan || !k_eff_host) return STEM_ERR_INVALID_ARG;
+  std::memcpy(k_eff_host, plan->p.k_eff.data(), plan->p.k_eff.size() * sizeof(int32_t));
+  return STEM_OK;
+}
+
+int stem_budget_table(const stem_config* cfg, int32_t* k_eff_host, int64_t capacity, int32_t* r_tot) {
+  int rc = validate(cfg);
+  if (rc != STEM_OK) return rc;
+  int64_t R = 0;
+  for (int b = 0; b < cfg->batch; ++b) {
+    const int64_t n = cfg->cu_seqlens_host[b + 1] - cfg->cu_seqlens_host[b];
+    const int64_t nb = (n + cfg->block - 1) / cfg->block;
+    const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb) / 1000;
+    for (int64_t r = 0; r < nb; ++r, ++R)
+      if (k_eff_host) {
+        if (R >= capacity) return STEM_ERR_INVALID_ARG;
+        k_eff_host[R] = budget_row(r + 1, nb, k_s, *cfg);
+      }
+  }
+  if (r_tot) *r_tot = (int32_t)R;
+  return STEM_OK;
+}
+
+int stem_last_launch_count(const stem_plan* plan) { return plan ? plan->p.last_launches : 0; }
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+static int check_ws(const Plan& p, const void* ws, size_t bytes) {
+  if (!ws || bytes < p.ws.total) return STEM_ERR_WORKSPACE;
+  if (((uintptr_t)ws & 255) != 0) return STEM_ERR_INVALID_ARG;
+  return STEM_OK;
+}
+
+static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
+
+int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* ws, size_t ws_bytes,
+               void* stream) {
+  if (!plan || !Q || !K || !V) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(M)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  uint8_t* w = (uint8_t*)ws;
+  cudaStream_t s = (cudaStream_t)stream;
+  p.last_launches = 0;
+  float* qbar = (float*)(w + p.ws.qbar);
+  float* kbar = (float*)(w + p.ws.kbar);
+  float* mv = (float*)(w + p.ws.mv);
+  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  if (M) {
+    rc = cuda_rc(launch_score_select(p, kFromPooled | kWriteMetric, qbar, kbar, mv, nullptr, M, nullptr, nullptr, s));
+    if (rc != STEM_OK) return rc;
+    p.last_launches++;
+  }
+  return STEM_OK;
+}
+
+int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t* sel_cnt, void* ws, size_t ws_bytes,
+                void* stream) {
+  if (!plan || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
+  if (misaligned(M) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  uint8_t* w = (uint8_t*)ws;
+  p.last_launches = 0;
+  const int mode = (M ? kFromMetric : kFromPooled) | kSelect;
+  rc = cuda_rc(launch_score_select(p, mode, (const float*)(w + p.ws.qbar), (const float*)(w + p.ws.kbar),
+                                   (const float*)(w + p.ws.mv), M, nullptr, sel_idx, sel_cnt, (cudaStream_t)stream));
+  if (rc == STEM_OK) p.last_launches++;
+  return rc;
+}
+
+int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, const int32_t* sel_idx,
+                        const int32_t* sel_cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  if (!plan || !Q || !K || !V || !O) return STEM_ERR_INVALID_ARG;
+  if ((sel_idx == nullptr) != (sel_cnt == nullptr)) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  p.last_launches = 0;
+  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, sel_idx, sel_cnt, O, lse, (int32_t*)((uint8_t*)ws + p.ws.status),
+                                       (cudaStream_t)stream));
+  if (rc == STEM_OK) p.last_launches++;
+  return rc;
+}
+
+int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
+                 int32_t* sel_cnt, float* lse, void* ws, size_t ws_bytes, void* stream) {
+  if (!plan || !Q || !K || !V || !O) return STEM_ERR_INVALID_ARG;
+  if ((sel_idx == nullptr) != (sel_cnt == nullptr)) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  uint8_t* w = (uint8_t*)ws;
+  cudaStream_t s = (cudaStream_t)stream;
+  float* qbar = (float*)(w + p.ws.qbar);
+  float* kbar = (float*)(w + p.ws.kbar);
+  float* mv = (float*)(w + p.ws.mv);
+  int32_t* idx = sel_idx ? sel_idx : (int32_t*)(w + p.ws.sel_idx);
+  int32_t* cnt = sel_cnt ? sel_cnt : (int32_t*)(w + p.ws.sel_cnt);
+  p.last_launches = 0;
+  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  rc = cuda_rc(launch_score_select(p, kFromPooled | kSelect, qbar, kbar, mv, nullptr, nullptr, idx, cnt, s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, idx, cnt, O, lse, (int32_t*)(w + p.ws.status), s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  return STEM_OK;
+}
+
+int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* detail) {
+  if (!plan || !ws) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t words[kStatusWords] = {0};
+  uint8_t* w = (uint8_t*)ws + p.ws.status;
+  if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  if (cudaMemcpy(words, w, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  if (detail) std::memcpy(detail, words, 4 * sizeof(int32_t));
+  if (words[0] != 0) {
+    cudaMemset(w, 0, sizeof(words));
+    return STEM_ERR_DEVICE_TIMEOUT;
+  }
+  return STEM_OK;
+}
+
+}  // extern "C"

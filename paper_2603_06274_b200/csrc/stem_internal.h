@@ -1,0 +1,84 @@
+// Internal declarations shared by the translation units of libstem (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "stem.h"
+
+namespace stem {
+
+constexpr int kHeadDim = 128;
+
+// Status words at the start of the workspace (int32 each).
+//   [0] code (0 = ok, 1 = a bounded wait gave up)   [1] CTA index   [2] role   [3] barrier id
+constexpr int kStatusWords = 8;
+
+// Device-side row tables, built once per plan.
+struct RowTables {
+  const int32_t* row_seq;      // [R_tot] sequence of global row R
+  const int32_t* row_r;        // [R_tot] row index inside its sequence
+  const int32_t* row_tok0;     // [R_tot] first packed token of the row's query block
+  const int32_t* row_ntok;     // [R_tot] valid tokens in that block (<= B)
+  const int32_t* row_keff;     // [R_tot] budget k_eff(r)
+  const int32_t* seq_tok0;     // [batch] first packed token of the sequence
+  const int32_t* seq_len;      // [batch]
+  const int32_t* seq_nblk;     // [batch]
+  const int32_t* seq_row_off;  // [batch] global row of the sequence's row 0
+  const int64_t* seq_m_off;    // [batch] offset of the sequence's square inside one head of M
+};
+
+// Where things live inside the caller's workspace (byte offsets, 256-aligned).
+struct WorkspaceLayout {
+  size_t status = 0;
+  size_t qbar = 0;     // fp32 [H_q, R_tot, d]
+  size_t kbar = 0;     // fp32 [H_kv, R_tot, d]
+  size_t mv = 0;       // fp32 [H_kv, R_tot]
+  size_t sel_idx = 0;  // int32 [H_q, R_tot, k_max]
+  size_t sel_cnt = 0;  // int32 [H_q, R_tot]
+  size_t total = 0;
+};
+
+struct Plan {
+  stem_config cfg{};
+  std::vector<int32_t> cu;  // host copy of cu_seqlens
+  int device = 0;
+  int sm_count = 0;
+  int32_t T = 0, R_tot = 0, k_max = 0, max_nblk = 0;
+  int64_t m_tot = 0;
+  int64_t selected_blocks = 0, causal_blocks = 0, selected_pairs = 0, causal_pairs = 0;
+  std::vector<int32_t> k_eff;  // host copy [R_tot]
+  float score_scale = 1.f, softmax_scale = 0.f;
+
+  // device blob
+  void* d_blob = nullptr;
+  RowTables rows{};
+  const int32_t* d_sel_tiles = nullptr;  // [n_sel_tiles][2] (sequence, first row) of the score/select tiles
+  int32_t n_sel_tiles = 0;
+  int32_t sel_rows_per_tile = 0;         // rows of one tile (all heads of a kv group ride together)
+  int32_t sel_nq = 0;                    // pooled query vectors per tile
+  const int32_t* d_work_sparse = nullptr;  // [n_items][2] (head, global row), attention work order
+  const int32_t* d_work_dense = nullptr;
+  int32_t n_items = 0;
+
+  WorkspaceLayout ws{};
+  mutable int last_launches = 0;
+};
+
+// Kernel launchers (each returns the cudaError_t of the launch).
+cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar,
+                        float* mv, cudaStream_t s);
+
+// mode bits for launch_score_select
+enum : int { kFromPooled = 1, kFromMetric = 2, kWriteMetric = 4, kSelect = 8 };
+cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar, const float* mv,
+                                const float* M_in, float* M_out, int32_t* sel_idx, int32_t* sel_cnt,
+                                cudaStream_t s);
+
+cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
+                                    const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,
+                                    int32_t* status, cudaStream_t s);
+
+}  // namespace stem

@@ -1,0 +1,98 @@
+"""Shared helpers for the GPU parity tests (device upload, oracle parameter mapping, comparisons)."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import stem_oracle as so
+from paper_2603_06274_b200 import workloads as wl
+
+# Tolerances of the attention output against the fp64 checker for bf16 inputs, same index set.
+ATTN_MAX_ABS = 2e-2
+ATTN_MEAN_ABS = 2e-3
+# A selection mismatch is tolerated only where the k-th / (k+1)-th metric values are this close.
+TIE_REL = 1e-3
+
+
+def to_dev(bits: np.ndarray) -> torch.Tensor:
+    """uint16 bf16 bit patterns -> CUDA bfloat16 tensor with the same bytes."""
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def from_dev_bf16(t: torch.Tensor) -> np.ndarray:
+    return t.float().cpu().numpy()
+
+
+def oracle_params(w: wl.Workload) -> so.StemParams:
+    return so.StemParams(block=w.block, budget_permille=w.budget_permille, k_start_blocks=w.k_start_blocks,
+                         mu_num=w.mu_num, mu_den=w.mu_den, stem_blocks=w.stem_blocks, local_blocks=w.local_blocks,
+                         min_blocks=w.min_blocks, beta=w.beta, score_scale=w.score_scale)
+
+
+def metric_views(M_flat: np.ndarray, nblk: np.ndarray):
+    """Split [H, sum nb^2] into per-sequence [H, nb, nb] views."""
+    out, off = [], 0
+    for nb in nblk:
+        nb = int(nb)
+        out.append(M_flat[:, off:off + nb * nb].reshape(M_flat.shape[0], nb, nb))
+        off += nb * nb
+    return out
+
+
+def compare_selection(idx_gpu, cnt_gpu, idx_ref, cnt_ref, M_ref, nblk, w: wl.Workload):
+    """Bit-exact comparison of index lists; rows that differ must be near-ties of the reference
+    metric at the top-k boundary (relative gap <= TIE_REL).  Returns the list of logged near-ties."""
+    assert np.array_equal(cnt_gpu, cnt_ref), "list lengths must equal the budget table"
+    diff_rows = np.argwhere((idx_gpu != idx_ref).any(axis=2))
+    logged = []
+    if len(diff_rows) == 0:
+        return logged
+    views = metric_views(M_ref, nblk)
+    row_off = np.concatenate([[0], np.cumsum(nblk)])
+    for h, R in diff_rows:
+        b = int(np.searchsorted(row_off, R, side="right") - 1)
+        r = int(R - row_off[b])
+        got = set(idx_gpu[h, R, :cnt_gpu[h, R]].tolist())
+        want = set(idx_ref[h, R, :cnt_ref[h, R]].tolist())
+        only_gpu, only_ref = got - want, want - got
+        assert len(only_gpu) == len(only_ref) and all(0 <= j <= r for j in got)
+        mrow = views[b][h, r]
+        # every swapped pair must straddle the boundary within the tie tolerance
+        top = max(float(mrow[j]) for j in only_ref)     # best block the GPU dropped
+        bottom = min(float(mrow[j]) for j in only_gpu)  # worst block the GPU took instead
+        gap = abs(top - bottom)
+        scale = max(abs(top), abs(bottom), 1e-30)
+        assert gap <= TIE_REL * scale, f"selection differs beyond a near-tie at head {h} row {R}: gap {gap}"
+        logged.append((int(h), int(R), gap / scale))
+    return logged
+
+
+def check_attention(o_gpu: np.ndarray, o_ref: np.ndarray, mask=None):
+    if mask is None:
+        mask = ~np.isnan(o_ref)
+    d = np.abs(o_gpu[mask].astype(np.float64) - o_ref[mask].astype(np.float64))
+    assert d.size > 0
+    assert np.isfinite(o_gpu[mask]).all()
+    assert d.max() <= ATTN_MAX_ABS, f"max abs {d.max()}"
+    assert d.mean() <= ATTN_MEAN_ABS, f"mean abs {d.mean()}"
+    return float(d.max()), float(d.mean())
+
+
+def sample_rows(hq: int, nblk: np.ndarray, k_s_rows, n_random: int, seed: int, full_heads=()):
+    """(head, global row) pairs: structural rows of every head plus seeded random rows."""
+    rng = np.random.default_rng(seed)
+    rows = set()
+    row_off = np.concatenate([[0], np.cumsum(nblk)])
+    for b, nb in enumerate(nblk):
+        nb = int(nb)
+        special = {0, nb // 2, nb - 1} | {min(nb - 1, max(0, int(x))) for x in k_s_rows}
+        for h in range(hq):
+            for r in special:
+                rows.add((h, int(row_off[b] + r)))
+        for h in full_heads:
+            for r in range(nb):
+                rows.add((h, int(row_off[b] + r)))
+    r_tot = int(row_off[-1])
+    for _ in range(n_random):
+        rows.add((int(rng.integers(hq)), int(rng.integers(r_tot))))
+    return np.array(sorted(rows), dtype=np.int32)
