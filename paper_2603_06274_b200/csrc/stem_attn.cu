@@ -52,7 +52,7 @@ struct Smem {
   static constexpr int s_full = q_empty + 16;
   static constexpr int p_ready = s_full + 8 * kNumSBuf;
   static constexpr int pv_done = p_ready + 8 * kNumSBuf;
-  static constexpr int drain = pv_done + 8;
+  static constexpr int drain = pv_done + 16;
   static constexpr int tmem_ptr = drain + 8;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
@@ -234,6 +234,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     for (int i = 0; i < 2; ++i) { mbar_init(bar(Smem::q_full, i), 1); mbar_init(bar(Smem::q_empty, i), 1); }
     for (int i = 0; i < kNumSBuf; ++i) { mbar_init(bar(Smem::s_full, i), 1); mbar_init(bar(Smem::p_ready, i), 128); }
     mbar_init(bar(Smem::pv_done, 0), 1);
+    mbar_init(bar(Smem::pv_done, 1), 1);
     mbar_init(bar(Smem::drain, 0), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -385,7 +386,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mma_ts(tmem_base + kOCol, p_tmem + k * 8, db, kIdescPV, (e > 0 || k > 0) ? 1u : 0u);
           }
           tc_commit(bar(Smem::kv_empty, slot));
-          tc_commit(bar(Smem::pv_done, 0));
+          tc_commit(bar(Smem::pv_done, (gblk + e) & 1));
           ++kv_cons;
         }
         gblk += n;
@@ -406,6 +407,19 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
     uint32_t gblk = 0;
     bool ok = true;
+    // P V products are counted globally (one per block, across items); product g arrives on
+    // pv_done[g & 1] as that barrier's phase g >> 1.  Completions are consumed strictly in order
+    // and never more than two behind the newest possible one, so a parity wait cannot alias.
+    uint32_t pv_waited = 0;
+    auto wait_pv_upto = [&](uint32_t target) -> bool {
+      bool good = true;
+      while (pv_waited < target && good) {
+        good = mbar_wait(bar(Smem::pv_done, pv_waited & 1), (pv_waited >> 1) & 1, ctx, kBarPvDone);
+        good = __all_sync(0xffffffffu, good);
+        ++pv_waited;
+      }
+      return good;
+    };
     for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
       const int h = a.work[2 * item], R = a.work[2 * item + 1];
       const int r = a.rows.row_r[R];
@@ -427,6 +441,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       for (int e = 0; e < n; ++e) {
         const uint32_t gb = gblk + e;
         const uint32_t sbuf = gb % kNumSBuf;
+        if (gb >= 1) { ok = wait_pv_upto(gb - 1); if (!ok) break; }  // long complete; keeps the count in step
         ok = mbar_wait(bar(Smem::s_full, sbuf), (gb / kNumSBuf) & 1, ctx, kBarSFull);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -449,8 +464,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           const bool grow = mx_c > m_run + kRescaleThreshold;
           if (__any_sync(0xffffffffu, grow)) {
             // O must hold every earlier P V product before it is rescaled
-            ok = mbar_wait(bar(Smem::pv_done, 0), (gb - 1) & 1, ctx, kBarPvDone);
-            ok = __all_sync(0xffffffffu, ok);
+            ok = wait_pv_upto(gb);
             if (!ok) break;
             tc_fence_after();
             const float alpha = grow ? fast_exp2(m_run - mx_c) : 1.f;
@@ -487,8 +501,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       if (!ok) break;
       gblk += n;
       // ---- epilogue: O / l -> bf16 -> global
-      ok = mbar_wait(bar(Smem::pv_done, 0), (gblk - 1) & 1, ctx, kBarPvDone);
-      ok = __all_sync(0xffffffffu, ok);
+      ok = wait_pv_upto(gblk);
       if (!ok) break;
       tc_fence_after();
       const float inv_l = 1.f / l_run;
