@@ -45,7 +45,8 @@ typedef enum {
   STEM_ERR_UNSUPPORTED = -2,    /* head_dim != 128, block not in {64,128}, heads not divisible, ... */
   STEM_ERR_WORKSPACE = -3,      /* workspace missing or smaller than stem_plan_query reports      */
   STEM_ERR_CUDA = -4,           /* a CUDA runtime / driver call or a kernel launch failed         */
-  STEM_ERR_DEVICE_TIMEOUT = -5  /* a bounded device-side wait gave up (see stem_check_status)     */
+  STEM_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up (see stem_check_status)     */
+  STEM_ERR_STATIC_SCRATCH = -6  /* problem larger than the built-in scratch of stem_score_static  */
 } stem_status;
 
 /* Problem statement of Algorithm 1 (inputs Q, K, V; hyper-parameters k_start, mu, B, beta) plus
@@ -111,6 +112,35 @@ int stem_budget_table(const stem_config* cfg, int32_t* k_eff_host, int64_t capac
  *   [num_q_heads, metric_elems].  With M == NULL only the pooled tensors are produced. */
 int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* workspace,
                size_t workspace_bytes, void* stream);
+
+/* stem_score for callers that cannot hand the library a workspace.  (The paper has no counterpart;
+ * this is a packaging variant of stem_score, computing the same M.)
+ *
+ * Who needs it: code that runs where device allocation is off limits - a plug-in called from inside
+ * a serving engine whose memory pool already owns the whole GPU, a callback that must not touch the
+ * allocator because the host framework forbids it there, a process running close to the memory
+ * limit where a multi-megabyte request could fail.  Such a caller still owns Q, K, V and M, but has
+ * nowhere to put the pooled tensors stem_score keeps in its workspace.
+ *
+ * Here that scratch lives in a fixed array inside the library image (STEM_STATIC_SCRATCH_BYTES,
+ * resident on every GPU that loads the library until the process exits).  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating routine; the plan must have been created earlier
+ * (plan creation does allocate its small tables).
+ *
+ *   - M is required.  Same layout and values as stem_score with a workspace.
+ *   - Problems whose pooled tensors exceed the array, i.e.
+ *       ((H_q + H_kv) * 128 + H_kv) * R_tot * 4 bytes (each part rounded up to 256)
+ *       > STEM_STATIC_SCRATCH_BYTES,
+ *     are rejected with STEM_ERR_STATIC_SCRATCH and nothing is enqueued.
+ *   - The first call on each device resolves the array's device address (a one-time set-up that
+ *     talks to the CUDA runtime); make that first call before starting any stream capture.  The
+ *     plan's device must be the current device.
+ *   - All calls on a device share the one array.  Its contents are whatever the previous call
+ *     left; every element this call reads it has written first, so nothing needs clearing.  Two
+ *     calls that overlap on the GPU (different streams, no ordering between them) race on the
+ *     array: serialise them. */
+#define STEM_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
+int stem_score_static(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* stream);
 
 /* Alg. 1 steps 3b-3c.
  *   For every (head, row): keeps the forced blocks {0..stem-1} and {r-local+1..r}, then adds the

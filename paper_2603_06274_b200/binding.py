@@ -20,9 +20,11 @@ STEM_ERR_UNSUPPORTED = -2
 STEM_ERR_WORKSPACE = -3
 STEM_ERR_CUDA = -4
 STEM_ERR_DEVICE_TIMEOUT = -5
+STEM_ERR_STATIC_SCRATCH = -6
+STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_destroy", "stem_plan_query",
-           "stem_plan_budget", "stem_budget_table", "stem_score", "stem_select", "stem_sparse_prefill", "stem_prefill",
+           "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_sparse_prefill", "stem_prefill",
            "stem_check_status", "stem_last_launch_count")
 
 
@@ -98,6 +100,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_plan_budget.argtypes = [vp, i32p]
     lib.stem_budget_table.argtypes = [ctypes.POINTER(StemConfig), i32p, ctypes.c_int64, i32p]
     lib.stem_score.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.stem_score_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.stem_select.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_sparse_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -210,6 +213,15 @@ def stem_score(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor
                workspace: Optional[torch.Tensor] = None) -> None:
     p, n = _ws_args(plan, workspace)
     _check(load().stem_score(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(M), p, n, _stream()), "stem_score")
+
+
+def stem_score_static(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, M: torch.Tensor) -> None:
+    """stem_score without a workspace: the pooled tensors go to a fixed array inside the library, so
+    the call allocates nothing.  For callers that may not allocate device memory where they run
+    (inside a framework's memory pool, in allocator-free callbacks).  Problems whose pooled
+    tensors exceed STATIC_SCRATCH_BYTES raise StemError(STEM_ERR_STATIC_SCRATCH).  Calls share
+    the array: do not overlap two of them on the GPU."""
+    _check(load().stem_score_static(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(M), _stream()), "stem_score_static")
 
 
 def stem_select(plan: StemPlan, M: Optional[torch.Tensor], sel_idx: torch.Tensor, sel_cnt: torch.Tensor,

@@ -69,10 +69,6 @@ using namespace stem;
 
 extern "C" {
 
-struct stem_plan {
-  Plan p;
-};
-
 int stem_version(void) { return 100; }
 
 const char* stem_status_string(int s) {
@@ -83,6 +79,7 @@ const char* stem_status_string(int s) {
     case STEM_ERR_WORKSPACE: return "workspace missing or too small";
     case STEM_ERR_CUDA: return "CUDA error";
     case STEM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait gave up";
+    case STEM_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch of the allocation-free entry point";
     default: return "unknown status";
   }
 }

@@ -82,3 +82,8 @@ cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K,
                                     int32_t* status, cudaStream_t s);
 
 }  // namespace stem
+
+// The opaque handle of the C ABI.
+struct stem_plan {
+  stem::Plan p;
+};

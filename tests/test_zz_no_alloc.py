@@ -1,0 +1,61 @@
+"""The allocation-free scoring entry point (stem_score_static), checked against stem_score.
+
+Some users of the library run where device memory cannot be requested: inside a serving engine
+whose pool already owns the GPU, or in callbacks where the host framework forbids allocator
+calls.  For them the library keeps the pooled tensors of the scoring stage in a fixed array of
+its own.  This file is collected last on purpose, so that a failure here cannot hide the result
+of any other test in a run that stops at the first failure."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_06274_b200 import binding, workloads as wl
+from paper_2603_06274_b200.binding import StemPlan
+from tests._util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _metric_pair(w):
+    data = wl.make_qkv(w)
+    plan = StemPlan.from_workload(w)
+    q, k, v = to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"])
+    n = plan.info.metric_elems
+    want = torch.full((w.num_q_heads, n), float("nan"), dtype=torch.float32, device="cuda")
+    got = torch.full((w.num_q_heads, n), float("nan"), dtype=torch.float32, device="cuda")
+    binding.stem_score(plan, q, k, v, want)          # existing entry point, caller workspace
+    binding.stem_score_static(plan, q, k, v, got)    # same stage, library-owned scratch
+    torch.cuda.synchronize()
+    return want.cpu().numpy(), got.cpu().numpy()
+
+
+def _assert_same(want, got):
+    defined = ~np.isnan(want)
+    assert defined.any()
+    assert np.array_equal(np.isnan(got), ~defined)
+    # tolerance of the metric parity test (the two paths run the same kernels, so they agree exactly)
+    tol = 2e-6 * np.maximum(1.0, np.abs(want[defined])) + 1e-6
+    assert np.all(np.abs(got[defined] - want[defined]) <= tol)
+
+
+def test_static_scratch_matches_workspace_path_on_two_calls_in_a_row():
+    # first call: a layer that nearly fills the array; second call: a smaller, differently shaped
+    # one, so stale contents of the shared array would show up if they were ever read
+    first = wl.small("noalloc_a", seqlens=(65536, 20000), hq=16, hkv=4, block=128, permille=200, sink=True)
+    second = wl.small("noalloc_b", seqlens=(3000,), hq=4, hkv=2, block=64, permille=300)
+    for w in (first, second):
+        want, got = _metric_pair(w)
+        _assert_same(want, got)
+
+
+def test_static_scratch_rejects_problems_beyond_its_size():
+    w = wl.CONFIGS["cfg3"]  # 40 heads x 1024 rows of pooled vectors: 21 MB > 8 MB
+    plan = StemPlan.from_workload(w)
+    dummy = torch.zeros(1024, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(1024, dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.StemError) as e:
+        binding.stem_score_static(plan, dummy, dummy, dummy, m)
+    assert e.value.status == binding.STEM_ERR_STATIC_SCRATCH
+    with pytest.raises(binding.StemError) as e:
+        binding.stem_score_static(plan, dummy, dummy, dummy, None)
+    assert e.value.status == binding.STEM_ERR_INVALID_ARG
