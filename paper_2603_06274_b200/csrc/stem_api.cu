@@ -45,6 +45,7 @@ static int validate(const stem_config* c) {
     return STEM_ERR_INVALID_ARG;
   if (!(c->beta == c->beta) || !(c->score_scale == c->score_scale) || !(c->softmax_scale == c->softmax_scale))
     return STEM_ERR_INVALID_ARG;
+  if (c->softmax_scale < 0.f) return STEM_ERR_INVALID_ARG;
   if (c->q_stride_tok % 8 || c->q_stride_head % 8 || c->kv_stride_tok % 8 || c->kv_stride_head % 8)
     return STEM_ERR_INVALID_ARG;
   if (c->q_stride_head < kHeadDim || c->kv_stride_head < kHeadDim) return STEM_ERR_INVALID_ARG;

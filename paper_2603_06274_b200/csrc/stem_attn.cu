@@ -1,18 +1,27 @@
 // Alg. 1 step 3d: exact causal softmax attention over the selected KV blocks, for sm_100a.
 //
-// One persistent CTA per SM walks a static share of the (head, query-block row) work items.
-// Per item it holds a 128-row Q tile in shared memory and streams the listed K / V blocks through
-// a ring of TMA-filled slots.  Both contractions run on tcgen05 tensor cores with fp32
-// accumulators in tensor memory (TMEM):
+// One persistent CTA per SM works on TWO (head, query-block row) items at a time ("slots" 0 and 1),
+// each with its own 128-row Q tile, its own index list and its own softmax warpgroup, so that the
+// tensor core computes one slot's products while the other slot's softmax runs.  Both contractions
+// use tcgen05 tensor cores with fp32 accumulators in tensor memory (TMEM):
 //     S = Q K_j^T          SS form, both operands K-major from 128B-swizzled shared memory
 //     O += P V_j           TS form, P (bf16) read from TMEM, V MN-major from shared memory
-// Warp roles (192 threads):
-//     warps 0-3  softmax: one thread per query row; tcgen05.ld S, online softmax in the log2
-//                domain with lazy rescaling of O, tcgen05.st P over S, final normalise + store
-//     warp 4     TMA producer (Q tiles double-buffered, K/V ring)
-//     warp 5     MMA issuer (one elected lane), owns the TMEM allocation
-// TMEM columns: three S/P buffers of 128 columns (so S_{j+2} can be issued before P_j V_j) and
-// one O accumulator of 128 columns.
+// Warp roles (384 threads):
+//     warps 0-3   softmax and epilogue of slot 0: one thread per query row; tcgen05.ld S, online
+//                 softmax in the log2 domain with lazy rescaling of O, tcgen05.st P over S; after
+//                 the item's last block O / l -> bf16 -> global memory
+//     warps 4-7   the same for slot 1
+//     warp 8      TMA producer of the K / V ring (one lane)
+//     warp 9      MMA issuer (one lane), owns the TMEM allocation
+//     warp 10     TMA producer of the Q tiles (one lane)
+// TMEM columns: S/P of slot 0, S/P of slot 1, O of slot 0, O of slot 1 (128 columns each).
+// The MMA issuer visits the slots alternately; a visit issues P V of the slot's previous block and
+// then Q K^T of its next block (P overwrites S, so the order inside a visit is fixed).  The K / V
+// producer walks the same visit sequence, so one shared ring serves both slots in order.  A slot's
+// items follow each other without a gap: Q K^T of the next item's first block is issued right
+// behind P V of the previous item's last block while the slot's softmax warps drain O.
+// Registers are re-balanced with setmaxnreg: the kernel must not spill, because with 227 KB of
+// shared memory in use almost no L1 is left for local memory.
 // Every mbarrier wait is bounded in time; a wait that gives up raises a CTA-wide abort flag,
 // records a status code and all roles fall through to the common teardown.
 #include <cuda.h>
@@ -26,38 +35,41 @@ namespace stem {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 384;
 constexpr int kTileM = 128;
 constexpr int kKvSlots = 5;
 constexpr int kSlotBytes = 32 * 1024;
 constexpr int kQBytes = 32 * 1024;
-constexpr int kNumSBuf = 3;
 constexpr int kTmemCols = 512;
-constexpr int kOCol = 384;
+constexpr int kOCol = 256;                               // O of slot X at kOCol + 128 X; S/P at 128 X
 constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;  // per wait
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
+constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // launch: 384 x 168; after: 256 x 208 + 128 x 88
 
-enum Role : int { kRoleSoftmax = 1, kRoleProducer = 2, kRoleMma = 3 };
-enum BarId : int { kBarKvFull = 1, kBarKvEmpty, kBarQFull, kBarQEmpty, kBarSFull, kBarPReady, kBarPvDone, kBarDrain };
+enum Role : int { kRoleSoftmax = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQProducer = 4 };
+enum BarId : int { kBarKvFull = 1, kBarKvEmpty, kBarQFull, kBarQEmpty, kBarSFull, kBarPReady, kBarOFull, kBarOFree,
+                   kBarDrain };
 
 struct Smem {
   // offsets from the 1024-aligned base
-  static constexpr int q = 0;
-  static constexpr int kv = q + 2 * kQBytes;
+  static constexpr int q = 0;                             // two Q tiles
+  static constexpr int kv = q + 2 * kQBytes;              // K / V ring
   static constexpr int bars = kv + kKvSlots * kSlotBytes;
   static constexpr int kv_full = bars;
   static constexpr int kv_empty = kv_full + 8 * kKvSlots;
   static constexpr int q_full = kv_empty + 8 * kKvSlots;
   static constexpr int q_empty = q_full + 16;
   static constexpr int s_full = q_empty + 16;
-  static constexpr int p_ready = s_full + 8 * kNumSBuf;
-  static constexpr int pv_done = p_ready + 8 * kNumSBuf;
-  static constexpr int drain = pv_done + 16;
+  static constexpr int p_ready = s_full + 16;
+  static constexpr int o_full = p_ready + 16;
+  static constexpr int o_free = o_full + 16;
+  static constexpr int drain = o_free + 16;
   static constexpr int tmem_ptr = drain + 8;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
 constexpr int kSmemBytes = Smem::total + 1024;  // slack for manual 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -88,26 +100,44 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
   return done;
 }
 
+// Non-blocking probe (try_wait may suspend the thread for a while; polling loops over several
+// barriers use this form).
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done;
+}
+
 struct Ctx {
   volatile int* abort_flag;  // shared memory
   int32_t* status;           // global memory status words
   int role;
 };
 
+__device__ __forceinline__ void raise_abort(const Ctx& c, int bar_id) {
+  *c.abort_flag = 1;
+  if (atomicCAS(c.status, 0, 1) == 0) {
+    c.status[1] = (int32_t)blockIdx.x;
+    c.status[2] = c.role;
+    c.status[3] = bar_id;
+  }
+}
+
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const Ctx& c, int bar_id, uint64_t limit_ns) {
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const Ctx& c, int bar_id, uint64_t limit_ns) {
   const uint64_t t0 = globaltimer();
   for (uint32_t spin = 0;; ++spin) {
     if (mbar_try(bar, parity)) return true;
     if ((spin & 31u) == 31u) {
       if (*c.abort_flag) return false;
       if (globaltimer() - t0 > limit_ns) {
-        *c.abort_flag = 1;
-        if (atomicCAS(c.status, 0, 1) == 0) {
-          c.status[1] = (int32_t)blockIdx.x;
-          c.status[2] = c.role;
-          c.status[3] = bar_id;
-        }
+        raise_abort(c, bar_id);
         return false;
       }
     }
@@ -174,6 +204,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -185,6 +223,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+
+template <int N>
+__device__ __forceinline__ void set_max_regs_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void set_max_regs_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // Shared-memory matrix descriptor for tcgen05.mma, 128-byte swizzle, sm_100 format (version 1).
@@ -216,6 +264,31 @@ struct AttnArgs {
   float scale_log2;
 };
 
+// Walks the items of one slot of this CTA: item i of the work order belongs to CTA i % gridDim.x,
+// slot (i / gridDim.x) % 2.  Items with an empty list are skipped (the slot's softmax warps zero
+// their output rows).
+struct ItemCursor {
+  int idx, step;
+  int h, R, r, n;
+  __device__ __forceinline__ void init(int slot) {
+    idx = (int)blockIdx.x + slot * (int)gridDim.x - 2 * (int)gridDim.x;
+    step = 2 * (int)gridDim.x;
+    n = 0;
+  }
+  // Moves to the next item with a non-empty list; false when the slot has no more items.
+  __device__ __forceinline__ bool next(const AttnArgs& a) {
+    for (idx += step; idx < a.n_items; idx += step) {
+      h = a.work[2 * idx];
+      R = a.work[2 * idx + 1];
+      r = a.rows.row_r[R];
+      n = a.sel_idx ? min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max) : r + 1;
+      if (n > 0) return true;
+    }
+    n = 0;
+    return false;
+  }
+};
+
 template <int BLK>
 __global__ void __launch_bounds__(kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -231,16 +304,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kKvSlots; ++i) { mbar_init(bar(Smem::kv_full, i), 1); mbar_init(bar(Smem::kv_empty, i), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(bar(Smem::q_full, i), 1); mbar_init(bar(Smem::q_empty, i), 1); }
-    for (int i = 0; i < kNumSBuf; ++i) { mbar_init(bar(Smem::s_full, i), 1); mbar_init(bar(Smem::p_ready, i), 128); }
-    mbar_init(bar(Smem::pv_done, 0), 1);
-    mbar_init(bar(Smem::pv_done, 1), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(Smem::q_full, i), 1);
+      mbar_init(bar(Smem::q_empty, i), 1);
+      mbar_init(bar(Smem::s_full, i), 1);
+      mbar_init(bar(Smem::p_ready, i), 4);   // one arrival per softmax warp
+      mbar_init(bar(Smem::o_full, i), 1);
+      mbar_init(bar(Smem::o_free, i), 4);    // one arrival per softmax warp
+    }
     mbar_init(bar(Smem::drain, 0), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 5) {
+  if (warp == 9) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + Smem::tmem_ptr),
                  "n"(kTmemCols)
                  : "memory");
@@ -257,179 +334,28 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   constexpr uint32_t kIdescPV = make_idesc(kHeadDim, 1);
   const bool dense = a.sel_idx == nullptr;
 
-  if (warp == 4) {
-    // ============================== TMA producer ==============================
-    Ctx ctx{abort_flag, a.status, kRoleProducer};
-    uint32_t kv_prod = 0;
-    int it = 0;
-    bool ok = true;
-    for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
-      const int h = a.work[2 * item], R = a.work[2 * item + 1];
-      const int r = a.rows.row_r[R];
-      const int seq_tok0 = a.rows.seq_tok0[a.rows.row_seq[R]];
-      const int q_tok0 = a.rows.row_tok0[R];
-      const int kvh = h / a.g;
-      int n = dense ? r + 1 : min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max);
-      if (n == 0) continue;
-      const int32_t* list = dense ? nullptr : a.sel_idx + ((int64_t)h * a.R_tot + R) * a.k_max;
-      const int qb = it & 1;
-      if (lane == 0) {
-        ok = mbar_wait(bar(Smem::q_empty, qb), ((it >> 1) & 1) ^ 1, ctx, kBarQEmpty);
-        if (ok) {
-          mbar_expect_tx(bar(Smem::q_full, qb), kQBytes);
-          tma_load_3d(smem_base + Smem::q + qb * kQBytes, &map_q, bar(Smem::q_full, qb), 0, h, q_tok0);
-          tma_load_3d(smem_base + Smem::q + qb * kQBytes + kTileM * 128, &map_q, bar(Smem::q_full, qb), 64, h, q_tok0);
-        }
-      }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      // load order: K0 K1 K2 V0 K3 V1 ... (the order the MMA warp consumes them in)
-      int32_t idx_reg = 0;  // lane l holds list[chunk*32 + l]
-      int chunk_loaded = -1;
-      for (int s = 0; s < n + 2 && ok; ++s) {
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          const int e = which == 0 ? s : s - 2;
-          if (which == 0 ? (s >= n) : (s < 2)) continue;
-          int j;
-          if (dense) {
-            j = e;
-          } else {
-            // V(e) trails K(e+2); both positions may sit in different 32-entry chunks of the list
-            const int chunk = e >> 5;
-            if (chunk != chunk_loaded) {
-              const int pos = chunk * 32 + lane;
-              idx_reg = pos < n ? list[pos] : 0;
-              chunk_loaded = chunk;
-            }
-            j = __shfl_sync(0xffffffffu, idx_reg, e & 31);
-            j = min(max(j, 0), r);
-          }
-          if (lane == 0 && ok) {
-            const uint32_t slot = kv_prod % kKvSlots;
-            ok = mbar_wait(bar(Smem::kv_empty, slot), ((kv_prod / kKvSlots) & 1) ^ 1, ctx, kBarKvEmpty);
-            if (ok) {
-              const CUtensorMap* m = which == 0 ? &map_k : &map_v;
-              const uint32_t dst = smem_base + Smem::kv + slot * kSlotBytes;
-              mbar_expect_tx(bar(Smem::kv_full, slot), kKvTileBytes);
-              tma_load_3d(dst, m, bar(Smem::kv_full, slot), 0, kvh, seq_tok0 + j * BLK);
-              tma_load_3d(dst + kHalfBytes, m, bar(Smem::kv_full, slot), 64, kvh, seq_tok0 + j * BLK);
-            }
-          }
-          ++kv_prod;
-          ok = __shfl_sync(0xffffffffu, ok, 0);
-        }
-      }
-      ++it;
-    }
-    if (!ok && lane == 0) {
-      // aborting: give copies already in flight a bounded time to land before the CTA exits
-      const uint32_t first = kv_prod > (uint32_t)kKvSlots ? kv_prod - kKvSlots : 0u;
-      for (uint32_t c = first; c < kv_prod; ++c) {
-        const uint64_t t0 = globaltimer();
-        while (!mbar_try(bar(Smem::kv_full, c % kKvSlots), (c / kKvSlots) & 1) && globaltimer() - t0 < 2000000ull) {}
-      }
-    }
-    __syncwarp();
-  } else if (warp == 5) {
-    // ============================== MMA issuer ==============================
-    Ctx ctx{abort_flag, a.status, kRoleMma};
-    uint32_t kv_cons = 0, gblk = 0;
-    int it = 0;
-    bool ok = true;
-    if (lane == 0) {
-      for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
-        const int h = a.work[2 * item], R = a.work[2 * item + 1];
-        const int r = a.rows.row_r[R];
-        const int n = dense ? r + 1 : min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max);
-        if (n == 0) continue;
-        const int qb = it & 1;
-        ok = mbar_wait(bar(Smem::q_full, qb), (it >> 1) & 1, ctx, kBarQFull);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t q_addr = smem_base + Smem::q + qb * kQBytes;
-        int s_issued = 0;
-        auto issue_s = [&](int e) -> bool {
-          const uint32_t slot = kv_cons % kKvSlots;
-          if (!mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull)) return false;
-          tc_fence_after();
-          const uint32_t k_addr = smem_base + Smem::kv + slot * kSlotBytes;
-          const uint32_t sbuf = (gblk + e) % kNumSBuf;
-          const uint32_t d_tmem = tmem_base + sbuf * 128;
-#pragma unroll
-          for (int k = 0; k < kHeadDim / 16; ++k) {
-            const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
-            const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
-            mma_ss(d_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
-          }
-          tc_commit(bar(Smem::kv_empty, slot));
-          tc_commit(bar(Smem::s_full, sbuf));
-          ++kv_cons;
-          if (++s_issued == n) tc_commit(bar(Smem::q_empty, qb));
-          return true;
-        };
-        for (int e = 0; e < min(2, n) && ok; ++e) ok = issue_s(e);
-        for (int e = 0; e < n && ok; ++e) {
-          const uint32_t sbuf = (gblk + e) % kNumSBuf;
-          ok = mbar_wait(bar(Smem::p_ready, sbuf), ((gblk + e) / kNumSBuf) & 1, ctx, kBarPReady);
-          if (!ok) break;
-          tc_fence_after();
-          if (e + 2 < n) { ok = issue_s(e + 2); if (!ok) break; }
-          const uint32_t slot = kv_cons % kKvSlots;
-          ok = mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t v_addr = smem_base + Smem::kv + slot * kSlotBytes;
-          const uint32_t p_tmem = tmem_base + sbuf * 128;
-#pragma unroll
-          for (int k = 0; k < BLK / 16; ++k) {
-            const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
-            mma_ts(tmem_base + kOCol, p_tmem + k * 8, db, kIdescPV, (e > 0 || k > 0) ? 1u : 0u);
-          }
-          tc_commit(bar(Smem::kv_empty, slot));
-          tc_commit(bar(Smem::pv_done, (gblk + e) & 1));
-          ++kv_cons;
-        }
-        gblk += n;
-        ++it;
-      }
-      if (!ok) {
-        // aborting: let the tensor-core work already issued finish (bounded) before TMEM is freed
-        tc_commit(bar(Smem::drain, 0));
-        const uint64_t t0 = globaltimer();
-        while (!mbar_try(bar(Smem::drain, 0), 0) && globaltimer() - t0 < 2000000ull) {}
-      }
-    }
-    __syncwarp();
-  } else {
-    // ============================== softmax + epilogue ==============================
+  if (warp < 8) {
+    // ============================== softmax of slot X ==============================
+    set_max_regs_inc<kRegsSoftmax>();
+    const int X = warp >> 2;
     Ctx ctx{abort_flag, a.status, kRoleSoftmax};
-    const int m = warp * 32 + lane;  // query row inside the tile == TMEM lane
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
-    uint32_t gblk = 0;
+    const int m = (warp & 3) * 32 + lane;  // query row inside the tile == TMEM lane
+    const uint32_t lane_addr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16);
+    const uint32_t s_addr = lane_addr + X * 128;
+    const uint32_t o_addr = lane_addr + kOCol + X * 128;
+    uint32_t blk = 0;   // blocks of this slot so far (phase of s_full / p_ready)
+    uint32_t ord = 0;   // non-empty items of this slot so far (phase of o_full / o_free)
     bool ok = true;
-    // P V products are counted globally (one per block, across items); product g arrives on
-    // pv_done[g & 1] as that barrier's phase g >> 1.  Completions are consumed strictly in order
-    // and never more than two behind the newest possible one, so a parity wait cannot alias.
-    uint32_t pv_waited = 0;
-    auto wait_pv_upto = [&](uint32_t target) -> bool {
-      bool good = true;
-      while (pv_waited < target && good) {
-        good = mbar_wait(bar(Smem::pv_done, pv_waited & 1), (pv_waited >> 1) & 1, ctx, kBarPvDone);
-        good = __all_sync(0xffffffffu, good);
-        ++pv_waited;
-      }
-      return good;
-    };
-    for (int item = blockIdx.x; item < a.n_items && ok; item += gridDim.x) {
+    for (int item = (int)blockIdx.x + X * (int)gridDim.x; item < a.n_items && ok; item += 2 * (int)gridDim.x) {
       const int h = a.work[2 * item], R = a.work[2 * item + 1];
       const int r = a.rows.row_r[R];
       const int q_tok0 = a.rows.row_tok0[R];
       const int ntok = a.rows.row_ntok[R];
       const int n = dense ? r + 1 : min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max);
       const bool row_valid = m < ntok;
-      __nv_bfloat16* o_row = a.O + ((int64_t)(q_tok0 + m) * a.Hq + h) * kHeadDim;
       if (n == 0) {
         if (row_valid) {
+          __nv_bfloat16* o_row = a.O + ((int64_t)(q_tok0 + m) * a.Hq + h) * kHeadDim;
 #pragma unroll
           for (int c = 0; c < 16; ++c) *(uint4*)(o_row + c * 8) = make_uint4(0, 0, 0, 0);
           if (a.lse) a.lse[(int64_t)h * a.T + q_tok0 + m] = -INFINITY;
@@ -438,78 +364,91 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       }
       const bool has_diag = dense || (a.sel_idx[((int64_t)h * a.R_tot + R) * a.k_max + n - 1] >= r);
       float m_run = -INFINITY, l_run = 0.f;
-      for (int e = 0; e < n; ++e) {
-        const uint32_t gb = gblk + e;
-        const uint32_t sbuf = gb % kNumSBuf;
-        if (gb >= 1) { ok = wait_pv_upto(gb - 1); if (!ok) break; }  // long complete; keeps the count in step
-        ok = mbar_wait(bar(Smem::s_full, sbuf), (gb / kNumSBuf) & 1, ctx, kBarSFull);
+      for (int e = 0; e < n; ++e, ++blk) {
+        // S of block e is complete; so is every earlier tensor-core operation of this slot,
+        // P V of block e-1 included (the commit behind Q K^T covers all earlier operations)
+        ok = mbar_wait(bar(Smem::s_full, X), blk & 1, ctx, kBarSFull);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
         float s[BLK];
 #pragma unroll
-        for (int c = 0; c < BLK / 32; ++c) tmem_ld32(lane_addr + sbuf * 128 + c * 32, &s[c * 32]);
+        for (int c = 0; c < BLK / 32; ++c) tmem_ld32(s_addr + c * 32, &s[c * 32]);
         tmem_ld_wait();
         if (e == n - 1 && has_diag) {
 #pragma unroll
           for (int c = 0; c < BLK; ++c) s[c] = (c <= m) ? s[c] : -INFINITY;
         }
-        float mx = s[0];
+        float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
 #pragma unroll
-        for (int c = 1; c < BLK; ++c) mx = fmaxf(mx, s[c]);
-        const float mx_c = mx * a.scale_log2;
+        for (int c = 6; c + 3 < BLK; c += 4) {
+          mx0 = max3(mx0, s[c], s[c + 1]);
+          mx1 = max3(mx1, s[c + 2], s[c + 3]);
+        }
+        const float mx_c = max3(mx0, mx1, fmaxf(s[BLK - 2], s[BLK - 1])) * a.scale_log2;
         if (e == 0) {
           m_run = mx_c;
         } else {
           const bool grow = mx_c > m_run + kRescaleThreshold;
           if (__any_sync(0xffffffffu, grow)) {
-            // O must hold every earlier P V product before it is rescaled
-            ok = wait_pv_upto(gb);
-            if (!ok) break;
-            tc_fence_after();
             const float alpha = grow ? fast_exp2(m_run - mx_c) : 1.f;
             if (grow) { m_run = mx_c; l_run *= alpha; }
 #pragma unroll
             for (int c = 0; c < kHeadDim / 32; ++c) {
               float o[32];
-              tmem_ld32(lane_addr + kOCol + c * 32, o);
+              tmem_ld32(o_addr + c * 32, o);
               tmem_ld_wait();
               uint32_t w[32];
 #pragma unroll
               for (int q = 0; q < 32; ++q) w[q] = __float_as_uint(o[q] * alpha);
-              tmem_st32(lane_addr + kOCol + c * 32, w);
+              tmem_st32(o_addr + c * 32, w);
             }
-            tmem_st_wait();
           }
         }
-        float sum = 0.f;
-        uint32_t pk[BLK / 2];
+        const float2 sc2 = make_float2(a.scale_log2, a.scale_log2);
+        const float2 nm2 = make_float2(-m_run, -m_run);
+        float2 sum_a = make_float2(0.f, 0.f), sum_b = make_float2(0.f, 0.f);
 #pragma unroll
-        for (int c = 0; c < BLK; c += 2) {
-          const float p0 = fast_exp2(fmaf(s[c], a.scale_log2, -m_run));
-          const float p1 = fast_exp2(fmaf(s[c + 1], a.scale_log2, -m_run));
-          sum += p0 + p1;
-          pk[c / 2] = pack_bf16(p0, p1);
+        for (int g = 0; g < BLK / 32; ++g) {
+          uint32_t pk[16];  // 32 probabilities as bf16 pairs = 16 TMEM columns
+#pragma unroll
+          for (int c = 0; c < 32; c += 4) {
+            const float2 x0 = __ffma2_rn(make_float2(s[g * 32 + c], s[g * 32 + c + 1]), sc2, nm2);
+            const float2 x1 = __ffma2_rn(make_float2(s[g * 32 + c + 2], s[g * 32 + c + 3]), sc2, nm2);
+            const float2 p0 = make_float2(fast_exp2(x0.x), fast_exp2(x0.y));
+            const float2 p1 = make_float2(fast_exp2(x1.x), fast_exp2(x1.y));
+            sum_a = __fadd2_rn(sum_a, p0);
+            sum_b = __fadd2_rn(sum_b, p1);
+            pk[c / 2] = pack_bf16(p0.x, p0.y);
+            pk[c / 2 + 1] = pack_bf16(p1.x, p1.y);
+          }
+          tmem_st16(s_addr + g * 16, pk);
         }
-        l_run += sum;
-#pragma unroll
-        for (int c = 0; c < BLK / 64; ++c) tmem_st32(lane_addr + sbuf * 128 + c * 32, &pk[c * 32]);
+        l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
         tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(bar(Smem::p_ready, sbuf));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(Smem::p_ready, X));
       }
       if (!ok) break;
-      gblk += n;
-      // ---- epilogue: O / l -> bf16 -> global
-      ok = wait_pv_upto(gblk);
+      // ---- epilogue: the item's last P V is complete -> O / l -> bf16 -> global memory
+      ok = mbar_wait(bar(Smem::o_full, X), ord & 1, ctx, kBarOFull);
+      ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
       const float inv_l = 1.f / l_run;
+      __nv_bfloat16* o_row = a.O + ((int64_t)(q_tok0 + m) * a.Hq + h) * kHeadDim;
 #pragma unroll
       for (int c = 0; c < kHeadDim / 32; ++c) {
         float o[32];
-        tmem_ld32(lane_addr + kOCol + c * 32, o);
+        tmem_ld32(o_addr + c * 32, o);
         tmem_ld_wait();
+        if (c == kHeadDim / 32 - 1) {
+          // O is in registers: P V of the slot's next item may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(Smem::o_free, X));
+        }
         if (row_valid) {
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -523,16 +462,198 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
       }
       if (a.lse && row_valid) a.lse[(int64_t)h * a.T + q_tok0 + m] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-      // all reads of O are complete (tmem_ld_wait) before this thread arrives on the next p_ready,
-      // which is what the next item's first P V (overwriting O) waits for.
-      tc_fence_before();
+      ++ord;
     }
+  } else {
+    set_max_regs_dec<kRegsOther>();
+    if (warp == 8 && lane == 0) {
+      // ============================== K / V producer ==============================
+      Ctx ctx{abort_flag, a.status, kRoleProducer};
+      struct KvSlot {
+        ItemCursor cur;
+        bool has, pend;
+        int e, j_next, pend_tok, pend_kvh, seq_tok0;
+        const int32_t* list;
+      };
+      auto enter = [&](KvSlot& s) {
+        s.has = s.cur.next(a);
+        s.e = 0;
+        if (s.has) {
+          s.seq_tok0 = a.rows.seq_tok0[a.rows.row_seq[s.cur.R]];
+          s.list = dense ? nullptr : a.sel_idx + ((int64_t)s.cur.h * a.R_tot + s.cur.R) * a.k_max;
+          s.j_next = dense ? 0 : s.list[0];
+        }
+      };
+      uint32_t kv_prod = 0;
+      auto load = [&](const CUtensorMap* map, int kvh, int tok) -> bool {
+        const uint32_t slot = kv_prod % kKvSlots;
+        if (!mbar_wait(bar(Smem::kv_empty, slot), ((kv_prod / kKvSlots) & 1) ^ 1, ctx, kBarKvEmpty)) return false;
+        const uint32_t dst = smem_base + Smem::kv + slot * kSlotBytes;
+        mbar_expect_tx(bar(Smem::kv_full, slot), kKvTileBytes);
+        tma_load_3d(dst, map, bar(Smem::kv_full, slot), 0, kvh, tok);
+        tma_load_3d(dst + kHalfBytes, map, bar(Smem::kv_full, slot), 64, kvh, tok);
+        ++kv_prod;
+        return true;
+      };
+      // One visit: V of the block whose K went out on the slot's previous visit, then K of the next block.
+      auto visit = [&](KvSlot& s) -> bool {
+        if (s.pend) {
+          s.pend = false;
+          if (!load(&map_v, s.pend_kvh, s.pend_tok)) return false;
+        }
+        if (s.has) {
+          const int j = min(max(s.j_next, 0), s.cur.r);
+          const int kvh = s.cur.h / a.g;
+          const int tok = s.seq_tok0 + j * BLK;
+          if (!load(&map_k, kvh, tok)) return false;
+          s.pend = true; s.pend_tok = tok; s.pend_kvh = kvh;
+          if (++s.e < s.cur.n) s.j_next = dense ? s.e : s.list[s.e];  // consumed on the slot's next visit
+          else enter(s);
+        }
+        return true;
+      };
+      KvSlot s0, s1;
+      s0.cur.init(0); s1.cur.init(1);
+      s0.pend = s1.pend = false;
+      enter(s0); enter(s1);
+      bool ok = true;
+      while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
+        ok = visit(s0);
+        if (ok) ok = visit(s1);
+      }
+      if (!ok) {
+        // aborting: give copies already in flight a bounded time to land before the CTA exits
+        const uint32_t first = kv_prod > (uint32_t)kKvSlots ? kv_prod - kKvSlots : 0u;
+        for (uint32_t c = first; c < kv_prod; ++c) {
+          const uint64_t t0 = globaltimer();
+          while (!mbar_try(bar(Smem::kv_full, c % kKvSlots), (c / kKvSlots) & 1) && globaltimer() - t0 < 2000000ull) {}
+        }
+      }
+    } else if (warp == 10 && lane == 0) {
+      // ============================== Q producer ==============================
+      Ctx ctx{abort_flag, a.status, kRoleQProducer};
+      ItemCursor c0, c1;
+      c0.init(0); c1.init(1);
+      bool has0 = c0.next(a), has1 = c1.next(a);
+      uint32_t ord0 = 0, ord1 = 0;
+      // Loads the slot's next Q tile as soon as the last Q K^T of its previous item has read the buffer.
+      auto try_load = [&](ItemCursor& cur, bool& has, uint32_t& ord, const int X) -> bool {
+        if (!has || !mbar_test(bar(Smem::q_empty, X), (ord & 1) ^ 1)) return false;
+        const int q_tok0 = a.rows.row_tok0[cur.R];
+        const uint32_t dst = smem_base + Smem::q + X * kQBytes;
+        mbar_expect_tx(bar(Smem::q_full, X), kQBytes);
+        tma_load_3d(dst, &map_q, bar(Smem::q_full, X), 0, cur.h, q_tok0);
+        tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, X), 64, cur.h, q_tok0);
+        ++ord;
+        has = cur.next(a);
+        return true;
+      };
+      bool ok = true;
+      uint64_t t0 = globaltimer();
+      uint32_t spin = 0;
+      while (ok && (has0 || has1)) {
+        const bool p0 = try_load(c0, has0, ord0, 0);
+        const bool p1 = try_load(c1, has1, ord1, 1);
+        if (p0 || p1) { t0 = globaltimer(); spin = 0; }
+        else if ((++spin & 31u) == 0u) {
+          if (*abort_flag) ok = false;
+          else if (globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); ok = false; }
+        }
+      }
+      if (!ok) {
+        // aborting: bounded wait for a Q copy that may still be in flight
+        const uint64_t t1 = globaltimer();
+        while (ord0 > 0 && !mbar_try(bar(Smem::q_full, 0), (ord0 - 1) & 1) && globaltimer() - t1 < 2000000ull) {}
+        while (ord1 > 0 && !mbar_try(bar(Smem::q_full, 1), (ord1 - 1) & 1) && globaltimer() - t1 < 4000000ull) {}
+      }
+    } else if (warp == 9 && lane == 0) {
+      // ============================== MMA issuer ==============================
+      Ctx ctx{abort_flag, a.status, kRoleMma};
+      struct MmaSlot {
+        ItemCursor cur;
+        bool has, pend, pend_first, pend_last;
+        int e;
+        uint32_t blk_pv, ord_qk, ord_pv;  // phases of p_ready, q_full, o_free
+      };
+      uint32_t kv_cons = 0;
+      auto visit = [&](MmaSlot& s, const int X) -> bool {
+        const uint32_t s_tmem = tmem_base + X * 128;
+        const uint32_t o_tmem = tmem_base + kOCol + X * 128;
+        if (s.pend) {
+          // ---- O_X (+)= P V of the block whose S went out on the slot's previous visit
+          if (!mbar_wait(bar(Smem::p_ready, X), s.blk_pv & 1, ctx, kBarPReady)) return false;
+          if (s.pend_first && !mbar_wait(bar(Smem::o_free, X), (s.ord_pv & 1) ^ 1, ctx, kBarOFree)) return false;
+          const uint32_t slot = kv_cons % kKvSlots;
+          if (!mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull)) return false;
+          tc_fence_after();
+          const uint32_t v_addr = smem_base + Smem::kv + slot * kSlotBytes;
+#pragma unroll
+          for (int k = 0; k < BLK / 16; ++k) {
+            const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
+            mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!s.pend_first || k > 0) ? 1u : 0u);
+          }
+          tc_commit(bar(Smem::kv_empty, slot));
+          ++kv_cons;
+          ++s.blk_pv;
+          if (s.pend_last) { tc_commit(bar(Smem::o_full, X)); ++s.ord_pv; }
+          s.pend = false;
+        }
+        if (s.has) {
+          // ---- S_X = Q K^T of the slot's next block (overwrites the P just consumed)
+          if (s.e == 0 && !mbar_wait(bar(Smem::q_full, X), s.ord_qk & 1, ctx, kBarQFull)) return false;
+          const uint32_t slot = kv_cons % kKvSlots;
+          if (!mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull)) return false;
+          tc_fence_after();
+          const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
+          const uint32_t k_addr = smem_base + Smem::kv + slot * kSlotBytes;
+#pragma unroll
+          for (int k = 0; k < kHeadDim / 16; ++k) {
+            const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
+            const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+            mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
+          }
+          tc_commit(bar(Smem::kv_empty, slot));
+          tc_commit(bar(Smem::s_full, X));
+          ++kv_cons;
+          s.pend = true;
+          s.pend_first = s.e == 0;
+          s.pend_last = s.e == s.cur.n - 1;
+          if (s.pend_last) {
+            tc_commit(bar(Smem::q_empty, X));
+            ++s.ord_qk;
+            s.has = s.cur.next(a);
+            s.e = 0;
+          } else {
+            ++s.e;
+          }
+        }
+        return true;
+      };
+      MmaSlot s0, s1;
+      s0.cur.init(0); s1.cur.init(1);
+      s0.has = s0.cur.next(a); s1.has = s1.cur.next(a);
+      s0.pend = s1.pend = s0.pend_first = s1.pend_first = s0.pend_last = s1.pend_last = false;
+      s0.e = s1.e = 0;
+      s0.blk_pv = s1.blk_pv = s0.ord_qk = s1.ord_qk = s0.ord_pv = s1.ord_pv = 0;
+      bool ok = true;
+      while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
+        ok = visit(s0, 0);
+        if (ok) ok = visit(s1, 1);
+      }
+      if (!ok) {
+        // aborting: let the tensor-core work already issued finish (bounded) before TMEM is freed
+        tc_commit(bar(Smem::drain, 0));
+        const uint64_t t0 = globaltimer();
+        while (!mbar_try(bar(Smem::drain, 0), 0) && globaltimer() - t0 < 2000000ull) {}
+      }
+    }
+    __syncwarp();
   }
 
   // ============================== teardown ==============================
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
   }
