@@ -11,9 +11,9 @@
 //                 softmax in the log2 domain with lazy rescaling of O, tcgen05.st P over S; after
 //                 the item's last block O / l -> bf16 -> global memory
 //     warps 4-7   the same for slot 1
-//     warp 8      TMA producer of the K / V ring (one lane)
-//     warp 9      MMA issuer (one lane), owns the TMEM allocation
-//     warp 10     TMA producer of the Q tiles (one lane)
+//     warp 8      TMA producer of the K / V ring (all lanes in lock step, one elected lane issues)
+//     warp 9      MMA issuer (likewise), owns the TMEM allocation
+//     warp 10     TMA producer of the Q tiles (likewise)
 // TMEM columns: S/P of slot 0, S/P of slot 1, O of slot 0, O of slot 1 (128 columns each).
 // The MMA issuer visits the slots alternately; a visit issues P V of the slot's previous block and
 // then Q K^T of its next block (P overwrites S, so the order inside a visit is fixed).  The K / V
@@ -110,6 +110,32 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(done)
       : "r"(bar), "r"(parity)
+      : "memory");
+  return done;
+}
+
+// Up to five independent probes issued back to back (so their shared-memory round trips overlap);
+// a disabled probe (en == 0) counts as complete.  Returns 1 when every enabled barrier phase is done.
+__device__ __forceinline__ uint32_t mbar_try5(uint32_t b0, uint32_t p0, uint32_t e0, uint32_t b1, uint32_t p1, uint32_t e1,
+                                              uint32_t b2, uint32_t p2, uint32_t e2, uint32_t b3, uint32_t p3, uint32_t e3,
+                                              uint32_t b4, uint32_t p4, uint32_t e4) {
+  uint32_t done;
+  asm volatile(
+      "{\n\t.reg .pred q0, q1, q2, q3, q4, r0, r1, r2, r3, r4;\n\t"
+      "setp.ne.b32 q0, %3, 0;\n\tsetp.ne.b32 q1, %6, 0;\n\tsetp.ne.b32 q2, %9, 0;\n\t"
+      "setp.ne.b32 q3, %12, 0;\n\tsetp.ne.b32 q4, %15, 0;\n\t"
+      "setp.eq.b32 r0, 0, 0;\n\tsetp.eq.b32 r1, 0, 0;\n\tsetp.eq.b32 r2, 0, 0;\n\t"
+      "setp.eq.b32 r3, 0, 0;\n\tsetp.eq.b32 r4, 0, 0;\n\t"
+      "@q0 mbarrier.try_wait.parity.shared::cta.b64 r0, [%1], %2;\n\t"
+      "@q1 mbarrier.try_wait.parity.shared::cta.b64 r1, [%4], %5;\n\t"
+      "@q2 mbarrier.try_wait.parity.shared::cta.b64 r2, [%7], %8;\n\t"
+      "@q3 mbarrier.try_wait.parity.shared::cta.b64 r3, [%10], %11;\n\t"
+      "@q4 mbarrier.try_wait.parity.shared::cta.b64 r4, [%13], %14;\n\t"
+      "and.pred r0, r0, r1;\n\tand.pred r2, r2, r3;\n\tand.pred r0, r0, r4;\n\tand.pred r0, r0, r2;\n\t"
+      "selp.u32 %0, 1, 0, r0;\n\t}"
+      : "=r"(done)
+      : "r"(b0), "r"(p0), "r"((uint32_t)e0), "r"(b1), "r"(p1), "r"((uint32_t)e1), "r"(b2), "r"(p2), "r"((uint32_t)e2),
+        "r"(b3), "r"(p3), "r"((uint32_t)e3), "r"(b4), "r"(p4), "r"((uint32_t)e4)
       : "memory");
   return done;
 }
@@ -224,7 +250,23 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+// Lane 0's value in every lane: marks a value the whole warp agrees on as warp-uniform.
+__device__ __forceinline__ int uni(int v) { return __shfl_sync(0xffffffffu, v, 0); }
 
 template <int N>
 __device__ __forceinline__ void set_max_regs_inc() {
@@ -266,7 +308,7 @@ struct AttnArgs {
 
 // Walks the items of one slot of this CTA: item i of the work order belongs to CTA i % gridDim.x,
 // slot (i / gridDim.x) % 2.  Items with an empty list are skipped (the slot's softmax warps zero
-// their output rows).
+// their output rows).  Used by whole warps in lock step (values are broadcast from lane 0).
 struct ItemCursor {
   int idx, step;
   int h, R, r, n;
@@ -278,10 +320,10 @@ struct ItemCursor {
   // Moves to the next item with a non-empty list; false when the slot has no more items.
   __device__ __forceinline__ bool next(const AttnArgs& a) {
     for (idx += step; idx < a.n_items; idx += step) {
-      h = a.work[2 * idx];
-      R = a.work[2 * idx + 1];
-      r = a.rows.row_r[R];
-      n = a.sel_idx ? min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max) : r + 1;
+      h = uni(a.work[2 * idx]);
+      R = uni(a.work[2 * idx + 1]);
+      r = uni(a.rows.row_r[R]);
+      n = a.sel_idx ? min(max(uni(a.sel_cnt[(int64_t)h * a.R_tot + R]), 0), a.k_max) : r + 1;
       if (n > 0) return true;
     }
     n = 0;
@@ -379,13 +421,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
           for (int c = 0; c < BLK; ++c) s[c] = (c <= m) ? s[c] : -INFINITY;
         }
-        float mx0 = max3(s[0], s[1], s[2]), mx1 = max3(s[3], s[4], s[5]);
+        float mx[8];
 #pragma unroll
-        for (int c = 6; c + 3 < BLK; c += 4) {
-          mx0 = max3(mx0, s[c], s[c + 1]);
-          mx1 = max3(mx1, s[c + 2], s[c + 3]);
+        for (int q = 0; q < 8; ++q) mx[q] = fmaxf(s[2 * q], s[2 * q + 1]);
+#pragma unroll
+        for (int c = 16; c < BLK; c += 16) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) mx[q] = max3(mx[q], s[c + 2 * q], s[c + 2 * q + 1]);
         }
-        const float mx_c = max3(mx0, mx1, fmaxf(s[BLK - 2], s[BLK - 1])) * a.scale_log2;
+        const float mx_c = fmaxf(max3(mx[0], mx[1], mx[2]), max3(mx[3], mx[4], max3(mx[5], mx[6], mx[7]))) * a.scale_log2;
         if (e == 0) {
           m_run = mx_c;
         } else {
@@ -465,8 +509,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       ++ord;
     }
   } else {
+    // The three issuing roles run with all 32 lanes in lock step on warp-uniform values (loads are
+    // broadcast through lane 0), so that descriptors, coordinates and barrier addresses live in
+    // uniform registers; only the TMA / MMA / commit instructions themselves are issued by one
+    // elected lane.
     set_max_regs_dec<kRegsOther>();
-    if (warp == 8 && lane == 0) {
+    if (warp == 8) {
       // ============================== K / V producer ==============================
       Ctx ctx{abort_flag, a.status, kRoleProducer};
       struct KvSlot {
@@ -479,19 +527,23 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         s.has = s.cur.next(a);
         s.e = 0;
         if (s.has) {
-          s.seq_tok0 = a.rows.seq_tok0[a.rows.row_seq[s.cur.R]];
+          s.seq_tok0 = uni(a.rows.seq_tok0[uni(a.rows.row_seq[s.cur.R])]);
           s.list = dense ? nullptr : a.sel_idx + ((int64_t)s.cur.h * a.R_tot + s.cur.R) * a.k_max;
-          s.j_next = dense ? 0 : s.list[0];
+          s.j_next = dense ? 0 : uni(s.list[0]);
         }
       };
-      uint32_t kv_prod = 0;
+      uint32_t ring = 0, ring_par = 0;  // next ring slot to fill and its phase
+      uint32_t kv_prod = 0;             // copies issued so far
       auto load = [&](const CUtensorMap* map, int kvh, int tok) -> bool {
-        const uint32_t slot = kv_prod % kKvSlots;
-        if (!mbar_wait(bar(Smem::kv_empty, slot), ((kv_prod / kKvSlots) & 1) ^ 1, ctx, kBarKvEmpty)) return false;
-        const uint32_t dst = smem_base + Smem::kv + slot * kSlotBytes;
-        mbar_expect_tx(bar(Smem::kv_full, slot), kKvTileBytes);
-        tma_load_3d(dst, map, bar(Smem::kv_full, slot), 0, kvh, tok);
-        tma_load_3d(dst + kHalfBytes, map, bar(Smem::kv_full, slot), 64, kvh, tok);
+        if (!__all_sync(0xffffffffu, mbar_wait(bar(Smem::kv_empty, ring), ring_par ^ 1, ctx, kBarKvEmpty))) return false;
+        const uint32_t dst = smem_base + Smem::kv + ring * kSlotBytes;
+        if (elect_one()) {
+          mbar_expect_tx(bar(Smem::kv_full, ring), kKvTileBytes);
+          tma_load_3d(dst, map, bar(Smem::kv_full, ring), 0, kvh, tok);
+          tma_load_3d(dst + kHalfBytes, map, bar(Smem::kv_full, ring), 64, kvh, tok);
+        }
+        __syncwarp();
+        if (++ring == kKvSlots) { ring = 0; ring_par ^= 1; }
         ++kv_prod;
         return true;
       };
@@ -507,7 +559,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           const int tok = s.seq_tok0 + j * BLK;
           if (!load(&map_k, kvh, tok)) return false;
           s.pend = true; s.pend_tok = tok; s.pend_kvh = kvh;
-          if (++s.e < s.cur.n) s.j_next = dense ? s.e : s.list[s.e];  // consumed on the slot's next visit
+          if (++s.e < s.cur.n) s.j_next = dense ? s.e : uni(s.list[s.e]);  // consumed on the slot's next visit
           else enter(s);
         }
         return true;
@@ -521,7 +573,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         ok = visit(s0);
         if (ok) ok = visit(s1);
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         // aborting: give copies already in flight a bounded time to land before the CTA exits
         const uint32_t first = kv_prod > (uint32_t)kKvSlots ? kv_prod - kKvSlots : 0u;
         for (uint32_t c = first; c < kv_prod; ++c) {
@@ -529,7 +581,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           while (!mbar_try(bar(Smem::kv_full, c % kKvSlots), (c / kKvSlots) & 1) && globaltimer() - t0 < 2000000ull) {}
         }
       }
-    } else if (warp == 10 && lane == 0) {
+    } else if (warp == 10) {
       // ============================== Q producer ==============================
       Ctx ctx{abort_flag, a.status, kRoleQProducer};
       ItemCursor c0, c1;
@@ -538,12 +590,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       uint32_t ord0 = 0, ord1 = 0;
       // Loads the slot's next Q tile as soon as the last Q K^T of its previous item has read the buffer.
       auto try_load = [&](ItemCursor& cur, bool& has, uint32_t& ord, const int X) -> bool {
-        if (!has || !mbar_test(bar(Smem::q_empty, X), (ord & 1) ^ 1)) return false;
-        const int q_tok0 = a.rows.row_tok0[cur.R];
+        if (!has || !uni((int)mbar_test(bar(Smem::q_empty, X), (ord & 1) ^ 1))) return false;
+        const int q_tok0 = uni(a.rows.row_tok0[cur.R]);
         const uint32_t dst = smem_base + Smem::q + X * kQBytes;
-        mbar_expect_tx(bar(Smem::q_full, X), kQBytes);
-        tma_load_3d(dst, &map_q, bar(Smem::q_full, X), 0, cur.h, q_tok0);
-        tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, X), 64, cur.h, q_tok0);
+        if (elect_one()) {
+          mbar_expect_tx(bar(Smem::q_full, X), kQBytes);
+          tma_load_3d(dst, &map_q, bar(Smem::q_full, X), 0, cur.h, q_tok0);
+          tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, X), 64, cur.h, q_tok0);
+        }
+        __syncwarp();
         ++ord;
         has = cur.next(a);
         return true;
@@ -556,71 +611,94 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const bool p1 = try_load(c1, has1, ord1, 1);
         if (p0 || p1) { t0 = globaltimer(); spin = 0; }
         else if ((++spin & 31u) == 0u) {
-          if (*abort_flag) ok = false;
-          else if (globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); ok = false; }
+          bool stop = *abort_flag != 0;
+          if (!stop && globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); stop = true; }
+          if (__any_sync(0xffffffffu, stop)) ok = false;
         }
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         // aborting: bounded wait for a Q copy that may still be in flight
         const uint64_t t1 = globaltimer();
         while (ord0 > 0 && !mbar_try(bar(Smem::q_full, 0), (ord0 - 1) & 1) && globaltimer() - t1 < 2000000ull) {}
         while (ord1 > 0 && !mbar_try(bar(Smem::q_full, 1), (ord1 - 1) & 1) && globaltimer() - t1 < 4000000ull) {}
       }
-    } else if (warp == 9 && lane == 0) {
+    } else if (warp == 9) {
       // ============================== MMA issuer ==============================
+      // One warp issues for both slots: two issuing warps (one per slot) measured 20 % slower.
       Ctx ctx{abort_flag, a.status, kRoleMma};
       struct MmaSlot {
         ItemCursor cur;
         bool has, pend, pend_first, pend_last;
         int e;
-        uint32_t blk_pv, ord_qk, ord_pv;  // phases of p_ready, q_full, o_free
+        uint32_t p_par, q_par, o_par;  // phase parities of p_ready, q_full, o_full / o_free
       };
-      uint32_t kv_cons = 0;
+      uint32_t ring = 0, ring_par = 0;  // next K / V ring slot to consume and its phase
+      // One visit.  Every barrier the visit depends on is probed up front in one go (independent
+      // shared-memory operations in flight together); only a failed probe falls back to the bounded waits.
       auto visit = [&](MmaSlot& s, const int X) -> bool {
         const uint32_t s_tmem = tmem_base + X * 128;
         const uint32_t o_tmem = tmem_base + kOCol + X * 128;
-        if (s.pend) {
-          // ---- O_X (+)= P V of the block whose S went out on the slot's previous visit
-          if (!mbar_wait(bar(Smem::p_ready, X), s.blk_pv & 1, ctx, kBarPReady)) return false;
-          if (s.pend_first && !mbar_wait(bar(Smem::o_free, X), (s.ord_pv & 1) ^ 1, ctx, kBarOFree)) return false;
-          const uint32_t slot = kv_cons % kKvSlots;
-          if (!mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull)) return false;
-          tc_fence_after();
-          const uint32_t v_addr = smem_base + Smem::kv + slot * kSlotBytes;
+        const bool do_pv = s.pend, do_qk = s.has;
+        const uint32_t slot_v = ring, par_v = ring_par;
+        uint32_t slot_k = ring, par_k = ring_par;
+        if (do_pv && ++slot_k == kKvSlots) { slot_k = 0; par_k ^= 1; }
+        const bool need_o = do_pv && s.pend_first, need_q = do_qk && s.e == 0;
+        const bool last = do_qk && s.e == s.cur.n - 1;
+        const uint32_t all_done =
+            mbar_try5(bar(Smem::p_ready, X), s.p_par, do_pv, bar(Smem::kv_full, slot_v), par_v, do_pv,
+                      bar(Smem::o_free, X), s.o_par ^ 1, need_o, bar(Smem::kv_full, slot_k), par_k, do_qk,
+                      bar(Smem::q_full, X), s.q_par, need_q);
+        if (!__all_sync(0xffffffffu, all_done != 0)) {
+          bool ok = true;
+          if (do_pv) ok = mbar_wait(bar(Smem::p_ready, X), s.p_par, ctx, kBarPReady) &&
+                          mbar_wait(bar(Smem::kv_full, slot_v), par_v, ctx, kBarKvFull);
+          if (ok && need_o) ok = mbar_wait(bar(Smem::o_free, X), s.o_par ^ 1, ctx, kBarOFree);
+          if (ok && do_qk) ok = mbar_wait(bar(Smem::kv_full, slot_k), par_k, ctx, kBarKvFull);
+          if (ok && need_q) ok = mbar_wait(bar(Smem::q_full, X), s.q_par, ctx, kBarQFull);
+          if (!__all_sync(0xffffffffu, ok)) return false;
+        }
+        tc_fence_after();
+        if (elect_one()) {
+          if (do_pv) {
+            // ---- O_X (+)= P V of the block whose S went out on the slot's previous visit
+            const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
 #pragma unroll
-          for (int k = 0; k < BLK / 16; ++k) {
-            const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
-            mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!s.pend_first || k > 0) ? 1u : 0u);
+            for (int k = 0; k < BLK / 16; ++k) {
+              const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
+              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!s.pend_first || k > 0) ? 1u : 0u);
+            }
+            tc_commit(bar(Smem::kv_empty, slot_v));
+            if (s.pend_last) tc_commit(bar(Smem::o_full, X));
           }
-          tc_commit(bar(Smem::kv_empty, slot));
-          ++kv_cons;
-          ++s.blk_pv;
-          if (s.pend_last) { tc_commit(bar(Smem::o_full, X)); ++s.ord_pv; }
+          if (do_qk) {
+            // ---- S_X = Q K^T of the slot's next block (overwrites the P just consumed)
+            const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
+            const uint32_t k_addr = smem_base + Smem::kv + slot_k * kSlotBytes;
+#pragma unroll
+            for (int k = 0; k < kHeadDim / 16; ++k) {
+              const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
+              const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+              mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(Smem::kv_empty, slot_k));
+            tc_commit(bar(Smem::s_full, X));
+            if (last) tc_commit(bar(Smem::q_empty, X));
+          }
+        }
+        __syncwarp();
+        if (do_pv) {
+          s.p_par ^= 1;
+          if (s.pend_last) s.o_par ^= 1;
           s.pend = false;
         }
-        if (s.has) {
-          // ---- S_X = Q K^T of the slot's next block (overwrites the P just consumed)
-          if (s.e == 0 && !mbar_wait(bar(Smem::q_full, X), s.ord_qk & 1, ctx, kBarQFull)) return false;
-          const uint32_t slot = kv_cons % kKvSlots;
-          if (!mbar_wait(bar(Smem::kv_full, slot), (kv_cons / kKvSlots) & 1, ctx, kBarKvFull)) return false;
-          tc_fence_after();
-          const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
-          const uint32_t k_addr = smem_base + Smem::kv + slot * kSlotBytes;
-#pragma unroll
-          for (int k = 0; k < kHeadDim / 16; ++k) {
-            const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
-            const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
-            mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
-          }
-          tc_commit(bar(Smem::kv_empty, slot));
-          tc_commit(bar(Smem::s_full, X));
-          ++kv_cons;
+        ring = slot_k; ring_par = par_k;
+        if (do_qk) {
+          if (++ring == kKvSlots) { ring = 0; ring_par ^= 1; }
           s.pend = true;
           s.pend_first = s.e == 0;
-          s.pend_last = s.e == s.cur.n - 1;
-          if (s.pend_last) {
-            tc_commit(bar(Smem::q_empty, X));
-            ++s.ord_qk;
+          s.pend_last = last;
+          if (last) {
+            s.q_par ^= 1;
             s.has = s.cur.next(a);
             s.e = 0;
           } else {
@@ -634,13 +712,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       s0.has = s0.cur.next(a); s1.has = s1.cur.next(a);
       s0.pend = s1.pend = s0.pend_first = s1.pend_first = s0.pend_last = s1.pend_last = false;
       s0.e = s1.e = 0;
-      s0.blk_pv = s1.blk_pv = s0.ord_qk = s1.ord_qk = s0.ord_pv = s1.ord_pv = 0;
+      s0.p_par = s1.p_par = s0.q_par = s1.q_par = s0.o_par = s1.o_par = 0;
       bool ok = true;
       while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
         ok = visit(s0, 0);
         if (ok) ok = visit(s1, 1);
       }
-      if (!ok) {
+      if (!ok && lane == 0) {
         // aborting: let the tensor-core work already issued finish (bounded) before TMEM is freed
         tc_commit(bar(Smem::drain, 0));
         const uint64_t t0 = globaltimer();
