@@ -107,6 +107,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_len(batch), seq_nblk(batch),
       seq_row_off(batch);
   std::vector<int64_t> seq_m_off(batch);
+  std::vector<int32_t> seq_kt_off(batch);
   int64_t m_off = 0;
   for (int b = 0; b < batch; ++b) {
     const int32_t n = p.cu[b + 1] - p.cu[b];
@@ -116,6 +117,8 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     seq_nblk[b] = nb;
     seq_row_off[b] = (int32_t)row_seq.size();
     seq_m_off[b] = m_off;
+    seq_kt_off[b] = p.kt_width;
+    p.kt_width += (nb + 63) / 64 * 64;
     m_off += (int64_t)nb * nb;
     p.max_nblk = std::max(p.max_nblk, nb);
     const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb) / 1000;
@@ -146,7 +149,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   // A tile holds at most 32 pooled query vectors and one fp32 metric row per vector in shared
   // memory, which bounds the number of blocks per sequence.
   const size_t ncols_pad = (size_t)(p.max_nblk + 63) / 64 * 64;
-  const size_t metric_smem_cap = 136 * 1024;  // what is left of 227 KB after the staging buffers
+  const size_t metric_smem_cap = 146 * 1024;  // what is left of 227 KB after the 80 KB of staging buffers
   int nq_cap = 32;
   while (nq_cap > g && (size_t)((nq_cap + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) nq_cap /= 2;
   if ((size_t)((std::max(1, nq_cap / g) * g + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) {
@@ -191,7 +194,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     size_t off = 0;
     p.ws.status = off; off = align_up(off + kStatusWords * 4, 256);
     p.ws.qbar = off;   off = align_up(off + (size_t)Hq * p.R_tot * kHeadDim * 4, 256);
-    p.ws.kbar = off;   off = align_up(off + (size_t)Hkv * p.R_tot * kHeadDim * 4, 256);
+    p.ws.kbar = off;   off = align_up(off + (size_t)Hkv * kHeadDim * p.kt_width * 4, 256);
     p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
     p.ws.sel_idx = off; off = align_up(off + (size_t)Hq * p.R_tot * p.k_max * 4, 256);
     p.ws.sel_cnt = off; off = align_up(off + (size_t)Hq * p.R_tot * 4, 256);
@@ -210,6 +213,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
                o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
                o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
                o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off),
+               o_seq_kt_off = push(blob, seq_kt_off),
                o_tiles = push(blob, tiles), o_ws = push(blob, work_sparse), o_wd = push(blob, work_dense);
   if (cudaMalloc(&p.d_blob, blob.size()) != cudaSuccess ||
       cudaMemcpy(p.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -229,6 +233,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.rows.seq_nblk = (const int32_t*)(d + o_seq_nblk);
   p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
+  p.rows.seq_kt_off = (const int32_t*)(d + o_seq_kt_off);
   p.d_sel_tiles = (const int32_t*)(d + o_tiles);
   p.d_work_sparse = (const int32_t*)(d + o_ws);
   p.d_work_dense = (const int32_t*)(d + o_wd);

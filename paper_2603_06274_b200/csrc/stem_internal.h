@@ -28,13 +28,14 @@ struct RowTables {
   const int32_t* seq_nblk;     // [batch]
   const int32_t* seq_row_off;  // [batch] global row of the sequence's row 0
   const int64_t* seq_m_off;    // [batch] offset of the sequence's square inside one head of M
+  const int32_t* seq_kt_off;   // [batch] first column of the sequence inside a row of Kbar^T (multiple of 64)
 };
 
 // Where things live inside the caller's workspace (byte offsets, 256-aligned).
 struct WorkspaceLayout {
   size_t status = 0;
   size_t qbar = 0;     // fp32 [H_q, R_tot, d]
-  size_t kbar = 0;     // fp32 [H_kv, R_tot, d]
+  size_t kbar = 0;     // fp32 [H_kv, d, kt_width]: Kbar transposed, block index contiguous
   size_t mv = 0;       // fp32 [H_kv, R_tot]
   size_t sel_idx = 0;  // int32 [H_q, R_tot, k_max]
   size_t sel_cnt = 0;  // int32 [H_q, R_tot]
@@ -47,6 +48,7 @@ struct Plan {
   int device = 0;
   int sm_count = 0;
   int32_t T = 0, R_tot = 0, k_max = 0, max_nblk = 0;
+  int32_t kt_width = 0;  // row length of Kbar^T: sum over sequences of N_blk rounded up to 64
   int64_t m_tot = 0;
   int64_t selected_blocks = 0, causal_blocks = 0, selected_pairs = 0, causal_pairs = 0;
   std::vector<int32_t> k_eff;  // host copy [R_tot]
@@ -68,12 +70,13 @@ struct Plan {
 };
 
 // Kernel launchers (each returns the cudaError_t of the launch).
-cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar,
+// qbar: [H_q, R_tot, d]; kbar_t: [H_kv, d, kt_width] (transposed for the scoring GEMM); mv: [H_kv, R_tot].
+cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t,
                         float* mv, cudaStream_t s);
 
 // mode bits for launch_score_select
 enum : int { kFromPooled = 1, kFromMetric = 2, kWriteMetric = 4, kSelect = 8 };
-cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar, const float* mv,
+cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar_t, const float* mv,
                                 const float* M_in, float* M_out, int32_t* sel_idx, int32_t* sel_cnt,
                                 cudaStream_t s);
 

@@ -35,8 +35,8 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
 template <int kBlock>
 __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                                                    const __nv_bfloat16* __restrict__ V, int64_t q_st, int64_t q_sh,
-                                                   int64_t kv_st, int64_t kv_sh, int Hq, int Hkv, int R_tot,
-                                                   RowTables rows, float* __restrict__ qbar, float* __restrict__ kbar,
+                                                   int64_t kv_st, int64_t kv_sh, int Hq, int Hkv, int R_tot, int kt_width,
+                                                   RowTables rows, float* __restrict__ qbar, float* __restrict__ kbar_t,
                                                    float* __restrict__ mv) {
   constexpr int kTokPerWarp = kBlock / 4;
   constexpr int kSteps = kTokPerWarp / 2;
@@ -85,8 +85,14 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
     __syncthreads();
     const int c = threadIdx.x;
     const float sum = (red[0][c] + red[1][c]) + (red[2][c] + red[3][c]);
-    float* out = (kind == 0 ? qbar : kbar) + ((int64_t)h * R_tot + R) * kHeadDim;
-    out[c] = sum / (float)ntok;
+    const float mean = sum / (float)ntok;
+    if (kind == 0) {
+      qbar[((int64_t)h * R_tot + R) * kHeadDim + c] = mean;
+    } else {
+      // Kbar is stored transposed ([H_kv, d, kt_width], block index contiguous) for the scoring GEMM
+      const int col = rows.seq_kt_off[rows.row_seq[R]] + rows.row_r[R];
+      kbar_t[((int64_t)h * kHeadDim + c) * kt_width + col] = mean;
+    }
   } else {
     float best = 0.f;  // squared norms are >= 0
 #pragma unroll
@@ -114,7 +120,7 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
 
 }  // namespace
 
-cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar, float* mv,
+cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t, float* mv,
                         cudaStream_t s) {
   const int slots = p.cfg.num_q_heads + 2 * p.cfg.num_kv_heads;
   const dim3 grid((unsigned)((int64_t)p.R_tot * slots));
@@ -123,12 +129,12 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
   auto v = (const __nv_bfloat16*)V;
   if (p.cfg.block == 128)
     pool_kernel<128><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
-                                          p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.rows,
-                                          qbar, kbar, mv);
+                                          p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
+                                          p.rows, qbar, kbar_t, mv);
   else
     pool_kernel<64><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
-                                         p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.rows,
-                                         qbar, kbar, mv);
+                                         p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
+                                         p.rows, qbar, kbar_t, mv);
   return cudaGetLastError();
 }
 

@@ -45,7 +45,7 @@ extern "C" int stem_score_static(const stem_plan* plan, const void* Q, const voi
 
   // Size check first: nothing is touched when the problem does not fit.
   const size_t qbar_bytes = align256((size_t)p.cfg.num_q_heads * p.R_tot * kHeadDim * sizeof(float));
-  const size_t kbar_bytes = align256((size_t)p.cfg.num_kv_heads * p.R_tot * kHeadDim * sizeof(float));
+  const size_t kbar_bytes = align256((size_t)p.cfg.num_kv_heads * kHeadDim * p.kt_width * sizeof(float));
   const size_t mv_bytes = align256((size_t)p.cfg.num_kv_heads * p.R_tot * sizeof(float));
   if (qbar_bytes + kbar_bytes + mv_bytes > (size_t)STEM_STATIC_SCRATCH_BYTES) return STEM_ERR_STATIC_SCRATCH;
 
