@@ -129,7 +129,8 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
  *
  *   - M is required.  Same layout and values as stem_score with a workspace.
  *   - Problems whose pooled tensors exceed the array, i.e.
- *       ((H_q + H_kv) * 128 + H_kv) * R_tot * 4 bytes (each part rounded up to 256)
+ *       (H_q * R_tot + H_kv * W) * 128 * 4 + H_kv * R_tot * 4 bytes (each part rounded up to 256),
+ *       W = sum over the sequences of N_blk rounded up to a multiple of 64,
  *       > STEM_STATIC_SCRATCH_BYTES,
  *     are rejected with STEM_ERR_STATIC_SCRATCH and nothing is enqueued.
  *   - The first call on each device resolves the array's device address (a one-time set-up that
