@@ -146,13 +146,16 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.causal_pairs *= Hq;
 
   // Score/select tiles: one CTA scores the g heads of a kv group for a run of consecutive rows.
-  // A tile holds at most 32 pooled query vectors and one fp32 metric row per vector in shared
-  // memory, which bounds the number of blocks per sequence.
-  const size_t ncols_pad = (size_t)(p.max_nblk + 63) / 64 * 64;
-  const size_t metric_smem_cap = 146 * 1024;  // what is left of 227 KB after the 80 KB of staging buffers
+  // A tile holds at most 32 pooled query vectors and one candidate list per vector in shared
+  // memory, which bounds the vectors per tile when the budget (list length) is large.
+  if (p.max_nblk > score_select_max_blocks()) {
+    delete sp;
+    return STEM_ERR_UNSUPPORTED;
+  }
+  const size_t list_bytes = score_select_list_bytes(p.k_max);
   int nq_cap = 32;
-  while (nq_cap > g && (size_t)((nq_cap + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) nq_cap /= 2;
-  if ((size_t)((std::max(1, nq_cap / g) * g + 7) / 8 * 8) * ncols_pad * 4 > metric_smem_cap) {
+  while (nq_cap > g && (size_t)((nq_cap + 7) / 8 * 8) * list_bytes > score_select_smem_budget()) nq_cap /= 2;
+  if ((size_t)((std::max(1, nq_cap / g) * g + 7) / 8 * 8) * list_bytes > score_select_smem_budget()) {
     delete sp;
     return STEM_ERR_UNSUPPORTED;
   }

@@ -74,6 +74,11 @@ struct Plan {
 cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t,
                         float* mv, cudaStream_t s);
 
+// Shared-memory needs of the score/select kernel, for sizing its tiles at plan creation.
+size_t score_select_list_bytes(int k_max);   // per pooled query vector
+size_t score_select_smem_budget();            // bytes available for the candidate lists of a tile
+int score_select_max_blocks();                // largest supported N_blk of a sequence
+
 // mode bits for launch_score_select
 enum : int { kFromPooled = 1, kFromMetric = 2, kWriteMetric = 4, kSelect = 8 };
 cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar_t, const float* mv,
