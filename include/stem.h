@@ -8,7 +8,8 @@
  *   stem_select          Alg. 1 steps 3b-3c: Token Position-Decay budget (Eq. 3, block units)
  *                        and per-row top-k with the forced stem / local blocks
  *   stem_sparse_prefill  Alg. 1 step 3d: exact causal softmax attention over the listed blocks
- *   stem_prefill         all of Algorithm 1 on one stream, no host synchronisation
+ *   stem_score_select    steps 1-3c in one call
+ *   stem_prefill         all of Algorithm 1, ordered on one stream, no host synchronisation
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned.
@@ -152,6 +153,13 @@ int stem_score_static(const stem_plan* plan, const void* Q, const void* K, const
 int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t* sel_cnt, void* workspace,
                 size_t workspace_bytes, void* stream);
 
+/* Alg. 1 steps 1-3c in one call: block-wise representations, Output-Aware Metric (Eq. 7), Token
+ * Position-Decay budget (Eq. 3) and top-k selection, without materialising M.
+ *   Same results as stem_score(M = NULL) followed by stem_select(M = NULL).
+ *   Writes sel_idx / sel_cnt; leaves the pooled tensors in the workspace. */
+int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const void* V, int32_t* sel_idx,
+                      int32_t* sel_cnt, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Alg. 1 step 3d.
  *   O[t,h,:] = softmax_k( Q[t,h].K[k,kv(h)] * softmax_scale ) V over the keys k of the listed
  *   blocks of t's row with position <= t.  sel_idx == NULL (with sel_cnt == NULL) means every
@@ -162,8 +170,8 @@ int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, con
                         const int32_t* sel_cnt, void* O, float* lse, void* workspace, size_t workspace_bytes,
                         void* stream);
 
-/* All of Algorithm 1: stem_score (without materialising M) -> stem_select -> stem_sparse_prefill on
- * `stream`.  sel_idx / sel_cnt are optional outputs (both NULL: lists stay in the workspace). */
+/* All of Algorithm 1: stem_score_select -> stem_sparse_prefill, ordered on `stream`, no host
+ * synchronisation.  sel_idx / sel_cnt are optional outputs (both NULL: lists stay in the workspace). */
 int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
                  int32_t* sel_cnt, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 

@@ -24,7 +24,7 @@ STEM_ERR_STATIC_SCRATCH = -6
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_destroy", "stem_plan_query",
-           "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_sparse_prefill", "stem_prefill",
+           "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_score_select", "stem_sparse_prefill", "stem_prefill",
            "stem_check_status", "stem_last_launch_count")
 
 
@@ -102,6 +102,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_score.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_score_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.stem_select.argtypes = [vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.stem_score_select.argtypes = [vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_sparse_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_check_status.argtypes = [vp, vp, vp, i32p]
@@ -228,6 +229,13 @@ def stem_select(plan: StemPlan, M: Optional[torch.Tensor], sel_idx: torch.Tensor
                 workspace: Optional[torch.Tensor] = None) -> None:
     p, n = _ws_args(plan, workspace)
     _check(load().stem_select(plan.handle, _ptr(M), _ptr(sel_idx), _ptr(sel_cnt), p, n, _stream()), "stem_select")
+
+
+def stem_score_select(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, sel_idx: torch.Tensor,
+                      sel_cnt: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> None:
+    p, n = _ws_args(plan, workspace)
+    _check(load().stem_score_select(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(sel_idx), _ptr(sel_cnt), p, n,
+                                    _stream()), "stem_score_select")
 
 
 def stem_sparse_prefill(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

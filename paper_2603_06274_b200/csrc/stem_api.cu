@@ -64,6 +64,13 @@ static size_t push(std::vector<uint8_t>& blob, const std::vector<T>& v) {
   return off;
 }
 
+// Frees everything a plan owns (also a half-built one).
+static void release_plan(stem_plan* sp) {
+  Plan& p = sp->p;
+  if (p.d_blob) cudaFree(p.d_blob);
+  delete sp;
+}
+
 }  // namespace stem
 
 using namespace stem;
@@ -246,8 +253,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
 
 int stem_plan_destroy(stem_plan* plan) {
   if (!plan) return STEM_ERR_INVALID_ARG;
-  if (plan->p.d_blob) cudaFree(plan->p.d_blob);
-  delete plan;
+  release_plan(plan);
   return STEM_OK;
 }
 
@@ -302,6 +308,20 @@ static int check_ws(const Plan& p, const void* ws, size_t bytes) {
 
 static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
 
+// Alg. 1 steps 1-3c: pooling, then scoring + selection of every tile, on one stream.
+// (Splitting the rows into phases and scoring the pooled ones on a second stream beside the
+// pooling of the rest was measured and dropped: at 0.2-0.3 ms per stage the cross-stream event
+// waits cost more than the overlap gains.)
+static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar,
+                                float* mv, int32_t* idx, int32_t* cnt, cudaStream_t s) {
+  int rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  rc = cuda_rc(launch_score_select(p, kFromPooled | kSelect, qbar, kbar, mv, nullptr, nullptr, idx, cnt, s));
+  if (rc == STEM_OK) p.last_launches++;
+  return rc;
+}
+
 int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* ws, size_t ws_bytes,
                void* stream) {
   if (!plan || !Q || !K || !V) return STEM_ERR_INVALID_ARG;
@@ -342,6 +362,20 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
   return rc;
 }
 
+int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const void* V, int32_t* sel_idx,
+                      int32_t* sel_cnt, void* ws, size_t ws_bytes, void* stream) {
+  if (!plan || !Q || !K || !V || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3))
+    return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  uint8_t* w = (uint8_t*)ws;
+  p.last_launches = 0;
+  return enqueue_score_select(p, Q, K, V, (float*)(w + p.ws.qbar), (float*)(w + p.ws.kbar), (float*)(w + p.ws.mv),
+                              sel_idx, sel_cnt, (cudaStream_t)stream);
+}
+
 int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, const int32_t* sel_idx,
                         const int32_t* sel_cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* stream) {
   if (!plan || !Q || !K || !V || !O) return STEM_ERR_INVALID_ARG;
@@ -373,12 +407,8 @@ int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void
   int32_t* idx = sel_idx ? sel_idx : (int32_t*)(w + p.ws.sel_idx);
   int32_t* cnt = sel_cnt ? sel_cnt : (int32_t*)(w + p.ws.sel_cnt);
   p.last_launches = 0;
-  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+  rc = enqueue_score_select(p, Q, K, V, qbar, kbar, mv, idx, cnt, s);
   if (rc != STEM_OK) return rc;
-  p.last_launches++;
-  rc = cuda_rc(launch_score_select(p, kFromPooled | kSelect, qbar, kbar, mv, nullptr, nullptr, idx, cnt, s));
-  if (rc != STEM_OK) return rc;
-  p.last_launches++;
   rc = cuda_rc(launch_sparse_attention(p, Q, K, V, idx, cnt, O, lse, (int32_t*)(w + p.ws.status), s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
