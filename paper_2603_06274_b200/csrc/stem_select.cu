@@ -15,12 +15,12 @@
 //
 // Selection is streaming, so a metric row never has to exist as a whole: every row keeps a short
 // list of (key, block) candidates in shared memory and a threshold tau.  A new metric value joins
-// the list only if its order-preserving key is above tau; when a list could overflow with the next
-// chunk it is cut back to the row's budget and tau rises to the smallest key kept.  Because blocks
-// arrive in ascending order, a later block with a key equal to tau can never displace a kept one
-// (ties go to the smaller block id), which is why the strict comparison loses nothing.  At the end
-// each row's list is cut to its budget, merged with the forced blocks through a bitmap and written
-// out in ascending order.
+// the list only if its order-preserving key is above tau; when a list runs full it is cut back
+// (keeping at least the row's budget of best entries), tau rises, and the values that did not fit
+// are offered again.  Because blocks arrive in ascending order, a later block with a key equal to
+// tau can never displace a kept one (ties go to the smaller block id), which is why the strict
+// comparison loses nothing.  At the end each row's list is cut to its budget, merged with the
+// forced blocks through a bitmap and written out in ascending order.
 #include "stem_internal.h"
 
 namespace stem {
