@@ -102,6 +102,22 @@ def dist_setup(n_gpus: int):
     return rank, world, local
 
 
+def max_over_ranks(x: float, world: int, device: str = "cuda") -> float:
+    """Largest value of x over the ranks of the default process group (x itself when there is one rank)."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_layer(rank: int) -> int:
+    """The path has no exchange step: rank r works on its own layer (seed offset r) of the workload."""
+    return rank
+
+
 def run_reference(args):
     """The CPU checker, as it stands, timed on this machine's host cores on a bounded sample."""
     rank, world, _ = dist_setup(args.gpus)
@@ -194,13 +210,6 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     def dev(bits):
         return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
 
@@ -215,10 +224,10 @@ def main():
             fn()
         e1.record()
         barrier()
-        return max_over_ranks(e0.elapsed_time(e1) / steps)
+        return max_over_ranks(e0.elapsed_time(e1) / steps, world)
 
     def bench_workload(w, steps, warmup, extras: bool):
-        data = wl.make_qkv(w, layer=rank)  # every rank draws its own layer
+        data = wl.make_qkv(w, layer=replica_layer(rank))  # every rank draws its own layer
         plan = pkg.StemPlan.from_workload(w)
         info = plan.info
         q, k, v = dev(data["q"]), dev(data["k"]), dev(data["v"])
