@@ -309,9 +309,9 @@ static int check_ws(const Plan& p, const void* ws, size_t bytes) {
 static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
 
 // Alg. 1 steps 1-3c: pooling, then scoring + selection of every tile, on one stream.
-// (Splitting the rows into phases and scoring the pooled ones on a second stream beside the
-// pooling of the rest was measured and dropped: at 0.2-0.3 ms per stage the cross-stream event
-// waits cost more than the overlap gains.)
+// (Two ways of overlapping the HBM-bound pooling with the FMA-bound scoring were measured and
+// dropped: phases on two streams lose more to cross-stream event waits than they gain, and one
+// persistent kernel with a shared ticket list leaves too few warps per SM to stream HBM.)
 static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar,
                                 float* mv, int32_t* idx, int32_t* cnt, cudaStream_t s) {
   int rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
