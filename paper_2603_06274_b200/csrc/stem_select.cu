@@ -264,19 +264,29 @@ __global__ void __launch_bounds__(kThreads, 2) score_select_kernel(TileArgs a) {
     if (from_pooled) {
       if (ch + 1 < n_chunks) load_chunk(ch + 1, (ch + 1) & 1);
       const float* kp_s = kt + (ch & 1) * kHeadDim * kChunk + (cg * 2 + ds) * 32 + kp * 2;
+      // packed fp32 FMAs (two vectors per instruction, same rounding as scalar FMAs): the loop is
+      // bound by instruction issue, not by the FMA pipe
+      float2 accp[4][2];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) { acc[i][0] = 0.f; acc[i][1] = 0.f; }
+      for (int i = 0; i < 4; ++i) { accp[i][0] = make_float2(0.f, 0.f); accp[i][1] = make_float2(0.f, 0.f); }
 #pragma unroll 8
       for (int dd = 0; dd < 64; ++dd) {
         const float4 qa = *(const float4*)(qp + dd * 64);
         const float4 qb = *(const float4*)(qp + dd * 64 + 4);
         const float2 kk = *(const float2*)(kp_s + dd * 128);
-        const float qv[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+        const float2 qpair[4] = {make_float2(qa.x, qa.y), make_float2(qa.z, qa.w), make_float2(qb.x, qb.y),
+                                 make_float2(qb.z, qb.w)};
+        const float2 kx = make_float2(kk.x, kk.x), ky = make_float2(kk.y, kk.y);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          acc[i][0] = fmaf(qv[i], kk.x, acc[i][0]);
-          acc[i][1] = fmaf(qv[i], kk.y, acc[i][1]);
+        for (int i = 0; i < 4; ++i) {
+          accp[i][0] = __ffma2_rn(qpair[i], kx, accp[i][0]);
+          accp[i][1] = __ffma2_rn(qpair[i], ky, accp[i][1]);
         }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc[2 * i][0] = accp[i][0].x; acc[2 * i + 1][0] = accp[i][0].y;
+        acc[2 * i][1] = accp[i][1].x; acc[2 * i + 1][1] = accp[i][1].y;
       }
       const float bias0 = (j0 < nblk) ? a.beta * mvb[j0] : 0.f;
       const float bias1 = (j0 + 1 < nblk) ? a.beta * mvb[j0 + 1] : 0.f;
