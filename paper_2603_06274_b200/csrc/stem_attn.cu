@@ -12,10 +12,11 @@
 //                 the item's last block O / l -> bf16 -> global memory
 //     warps 4-7   the same for slot 1
 //     warp 8      TMA producer of the K / V ring (all lanes in lock step, one elected lane issues)
-//     warp 9      MMA issuer (likewise), owns the TMEM allocation
+//     warp 9      MMA scheduler (likewise): waits on the barriers of each visit, owns the TMEM allocation
 //     warp 10     TMA producer of the Q tiles (likewise)
+//     warp 11     MMA issuer (likewise): issues the visits the scheduler hands over
 // TMEM columns: S/P of slot 0, S/P of slot 1, O of slot 0, O of slot 1 (128 columns each).
-// The MMA issuer visits the slots alternately; a visit issues P V of the slot's previous block and
+// The MMA scheduler visits the slots alternately; a visit issues P V of the slot's previous block and
 // then Q K^T of its next block (P overwrites S, so the order inside a visit is fixed).  The K / V
 // producer walks the same visit sequence, so one shared ring serves both slots in order.  A slot's
 // items follow each other without a gap: Q K^T of the next item's first block is issued right
@@ -41,6 +42,7 @@ constexpr int kKvSlots = 5;
 constexpr int kSlotBytes = 32 * 1024;
 constexpr int kQBytes = 32 * 1024;
 constexpr int kTmemCols = 512;
+constexpr int kCmdSlots = 4;
 constexpr int kOCol = 256;                               // O of slot X at kOCol + 128 X; S/P at 128 X
 constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;  // per wait
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
@@ -48,7 +50,10 @@ constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // launch: 384 x 168; after:
 
 enum Role : int { kRoleSoftmax = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQProducer = 4 };
 enum BarId : int { kBarKvFull = 1, kBarKvEmpty, kBarQFull, kBarQEmpty, kBarSFull, kBarPReady, kBarOFull, kBarOFree,
-                   kBarDrain };
+                   kBarDrain, kBarCmdFull, kBarCmdEmpty };
+// One visit of the MMA issuer as a command word.
+enum Cmd : uint32_t { kCmdPv = 1u, kCmdQk = 2u, kCmdPvFirst = 4u, kCmdPvLast = 8u, kCmdQkLast = 16u, kCmdSlot1 = 32u,
+                      kCmdExit = 0x80000000u };
 
 struct Smem {
   // offsets from the 1024-aligned base
@@ -64,7 +69,10 @@ struct Smem {
   static constexpr int o_full = p_ready + 16;
   static constexpr int o_free = o_full + 16;
   static constexpr int drain = o_free + 16;
-  static constexpr int tmem_ptr = drain + 8;
+  static constexpr int cmd_full = drain + 8;               // scheduler -> issuer command ring
+  static constexpr int cmd_empty = cmd_full + 8 * kCmdSlots;
+  static constexpr int cmd_word = cmd_empty + 8 * kCmdSlots;
+  static constexpr int tmem_ptr = cmd_word + 4 * kCmdSlots;
   static constexpr int abort_flag = tmem_ptr + 4;
   static constexpr int total = abort_flag + 4;
 };
@@ -355,6 +363,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       mbar_init(bar(Smem::o_free, i), 4);    // one arrival per softmax warp
     }
     mbar_init(bar(Smem::drain, 0), 1);
+    for (int i = 0; i < kCmdSlots; ++i) { mbar_init(bar(Smem::cmd_full, i), 1); mbar_init(bar(Smem::cmd_empty, i), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -623,9 +632,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         while (ord1 > 0 && !mbar_try(bar(Smem::q_full, 1), (ord1 - 1) & 1) && globaltimer() - t1 < 4000000ull) {}
       }
     } else if (warp == 9) {
-      // ============================== MMA issuer ==============================
-      // One warp issues for both slots: two issuing warps (one per slot) measured 20 % slower.
+      // ============================== MMA scheduler ==============================
+      // Decides what the tensor core does next and checks that it can be done (P ready, K / V and
+      // Q landed, O drained); the MMAs themselves are issued by warp 11 from a small command ring.
+      // tcgen05.mma issue blocks while the short tensor queue is full, so a warp that both waits on
+      // barriers and issues leaves the tensor core idle during its own book-keeping.
       Ctx ctx{abort_flag, a.status, kRoleMma};
+      volatile uint32_t* cmd_word = (volatile uint32_t*)(smem_gen + Smem::cmd_word);
+      uint32_t ci = 0, cpar = 0;  // next command slot and its phase
       struct MmaSlot {
         ItemCursor cur;
         bool has, pend, pend_first, pend_last;
@@ -636,8 +650,6 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       // One visit.  Every barrier the visit depends on is probed up front in one go (independent
       // shared-memory operations in flight together); only a failed probe falls back to the bounded waits.
       auto visit = [&](MmaSlot& s, const int X) -> bool {
-        const uint32_t s_tmem = tmem_base + X * 128;
-        const uint32_t o_tmem = tmem_base + kOCol + X * 128;
         const bool do_pv = s.pend, do_qk = s.has;
         const uint32_t slot_v = ring, par_v = ring_par;
         uint32_t slot_k = ring, par_k = ring_par;
@@ -657,35 +669,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           if (ok && need_q) ok = mbar_wait(bar(Smem::q_full, X), s.q_par, ctx, kBarQFull);
           if (!__all_sync(0xffffffffu, ok)) return false;
         }
-        tc_fence_after();
-        if (elect_one()) {
-          if (do_pv) {
-            // ---- O_X (+)= P V of the block whose S went out on the slot's previous visit
-            const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
-#pragma unroll
-            for (int k = 0; k < BLK / 16; ++k) {
-              const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
-              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!s.pend_first || k > 0) ? 1u : 0u);
-            }
-            tc_commit(bar(Smem::kv_empty, slot_v));
-            if (s.pend_last) tc_commit(bar(Smem::o_full, X));
-          }
-          if (do_qk) {
-            // ---- S_X = Q K^T of the slot's next block (overwrites the P just consumed)
-            const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
-            const uint32_t k_addr = smem_base + Smem::kv + slot_k * kSlotBytes;
-#pragma unroll
-            for (int k = 0; k < kHeadDim / 16; ++k) {
-              const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
-              const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
-              mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
-            }
-            tc_commit(bar(Smem::kv_empty, slot_k));
-            tc_commit(bar(Smem::s_full, X));
-            if (last) tc_commit(bar(Smem::q_empty, X));
-          }
+        // everything the visit needs is in place: hand it to the issuing warp
+        if (!__all_sync(0xffffffffu, mbar_wait(bar(Smem::cmd_empty, ci), cpar ^ 1, ctx, kBarCmdEmpty))) return false;
+        if (lane == 0) {
+          cmd_word[ci] = (do_pv ? kCmdPv : 0u) | (do_qk ? kCmdQk : 0u) | (s.pend_first ? kCmdPvFirst : 0u) |
+                         (s.pend_last ? kCmdPvLast : 0u) | (last ? kCmdQkLast : 0u) | (X ? kCmdSlot1 : 0u) |
+                         (slot_v << 8) | (slot_k << 12);
+          mbar_arrive(bar(Smem::cmd_full, ci));  // release: the word and everything observed above
         }
         __syncwarp();
+        if (++ci == kCmdSlots) { ci = 0; cpar ^= 1; }
         if (do_pv) {
           s.p_par ^= 1;
           if (s.pend_last) s.o_par ^= 1;
@@ -717,6 +710,60 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
         ok = visit(s0, 0);
         if (ok) ok = visit(s1, 1);
+      }
+      // tell the issuing warp that nothing follows (also when aborting: its own waits are bounded too)
+      if (__all_sync(0xffffffffu, mbar_wait(bar(Smem::cmd_empty, ci), cpar ^ 1, ctx, kBarCmdEmpty)) && lane == 0) {
+        cmd_word[ci] = kCmdExit;
+        mbar_arrive(bar(Smem::cmd_full, ci));
+      }
+    } else if (warp == 11) {
+      // ============================== MMA issuer ==============================
+      // Executes the scheduler's commands in order: O_X (+)= P V of a block, then S_X = Q K^T of the
+      // slot's next block (which overwrites the P just consumed), with the commits that publish them.
+      Ctx ctx{abort_flag, a.status, kRoleMma};
+      volatile uint32_t* cmd_word = (volatile uint32_t*)(smem_gen + Smem::cmd_word);
+      uint32_t ci = 0, cpar = 0;
+      bool ok = true;
+      for (;;) {
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(Smem::cmd_full, ci), cpar, ctx, kBarCmdFull));
+        if (!ok) break;
+        const uint32_t cmd = (uint32_t)uni((int)cmd_word[ci]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(Smem::cmd_empty, ci));
+        if (++ci == kCmdSlots) { ci = 0; cpar ^= 1; }
+        if (cmd & kCmdExit) break;
+        const uint32_t X = (cmd & kCmdSlot1) ? 1u : 0u;
+        const uint32_t slot_v = (cmd >> 8) & 15u, slot_k = (cmd >> 12) & 15u;
+        const uint32_t s_tmem = tmem_base + X * 128;
+        const uint32_t o_tmem = tmem_base + kOCol + X * 128;
+        tc_fence_after();
+        if (elect_one()) {
+          if (cmd & kCmdPv) {
+            const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
+            const uint32_t first = (cmd & kCmdPvFirst) ? 1u : 0u;
+#pragma unroll
+            for (int k = 0; k < BLK / 16; ++k) {
+              const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
+              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!first || k > 0) ? 1u : 0u);
+            }
+            tc_commit(bar(Smem::kv_empty, slot_v));
+            if (cmd & kCmdPvLast) tc_commit(bar(Smem::o_full, X));
+          }
+          if (cmd & kCmdQk) {
+            const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
+            const uint32_t k_addr = smem_base + Smem::kv + slot_k * kSlotBytes;
+#pragma unroll
+            for (int k = 0; k < kHeadDim / 16; ++k) {
+              const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
+              const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+              mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
+            }
+            tc_commit(bar(Smem::kv_empty, slot_k));
+            tc_commit(bar(Smem::s_full, X));
+            if (cmd & kCmdQkLast) tc_commit(bar(Smem::q_empty, X));
+          }
+        }
+        __syncwarp();
       }
       if (!ok && lane == 0) {
         // aborting: let the tensor-core work already issued finish (bounded) before TMEM is freed
