@@ -12,9 +12,11 @@
 //                 the item's last block O / l -> bf16 -> global memory
 //     warps 4-7   the same for slot 1
 //     warp 8      TMA producer of the K / V ring (all lanes in lock step, one elected lane issues)
-//     warp 9      MMA scheduler (likewise): waits on the barriers of each visit, owns the TMEM allocation
+//     warp 9      MMA scheduler (likewise): checks ahead of time that K / V, Q and O of each visit are in
+//                 place and queues the visit for the issuer; owns the TMEM allocation
 //     warp 10     TMA producer of the Q tiles (likewise)
-//     warp 11     MMA issuer (likewise): issues the visits the scheduler hands over
+//     warp 11     MMA issuer (likewise): waits for P of the queued visit and issues its MMAs; P V starts on
+//                 the leading key columns while the softmax still works on the last 32
 // TMEM columns: S/P of slot 0, S/P of slot 1, O of slot 0, O of slot 1 (128 columns each).
 // The MMA scheduler visits the slots alternately; a visit issues P V of the slot's previous block and
 // then Q K^T of its next block (P overwrites S, so the order inside a visit is fixed).  The K / V
@@ -50,9 +52,10 @@ constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // launch: 384 x 168; after:
 
 enum Role : int { kRoleSoftmax = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQProducer = 4 };
 enum BarId : int { kBarKvFull = 1, kBarKvEmpty, kBarQFull, kBarQEmpty, kBarSFull, kBarPReady, kBarOFull, kBarOFree,
-                   kBarDrain, kBarCmdFull, kBarCmdEmpty };
+                   kBarDrain, kBarCmdFull, kBarCmdEmpty, kBarPEarly };
 // One visit of the MMA issuer as a command word.
 enum Cmd : uint32_t { kCmdPv = 1u, kCmdQk = 2u, kCmdPvFirst = 4u, kCmdPvLast = 8u, kCmdQkLast = 16u, kCmdSlot1 = 32u,
+                      kCmdPPar = 64u,  // phase parity of p_ready the P V of this visit waits for
                       kCmdExit = 0x80000000u };
 
 struct Smem {
@@ -66,7 +69,8 @@ struct Smem {
   static constexpr int q_empty = q_full + 16;
   static constexpr int s_full = q_empty + 16;
   static constexpr int p_ready = s_full + 16;
-  static constexpr int o_full = p_ready + 16;
+  static constexpr int p_early = p_ready + 16;            // all of P but its last 32 key columns stored
+  static constexpr int o_full = p_early + 16;
   static constexpr int o_free = o_full + 16;
   static constexpr int drain = o_free + 16;
   static constexpr int cmd_full = drain + 8;               // scheduler -> issuer command ring
@@ -122,28 +126,24 @@ __device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
   return done;
 }
 
-// Up to five independent probes issued back to back (so their shared-memory round trips overlap);
+// Up to four independent probes issued back to back (so their shared-memory round trips overlap);
 // a disabled probe (en == 0) counts as complete.  Returns 1 when every enabled barrier phase is done.
-__device__ __forceinline__ uint32_t mbar_try5(uint32_t b0, uint32_t p0, uint32_t e0, uint32_t b1, uint32_t p1, uint32_t e1,
-                                              uint32_t b2, uint32_t p2, uint32_t e2, uint32_t b3, uint32_t p3, uint32_t e3,
-                                              uint32_t b4, uint32_t p4, uint32_t e4) {
+__device__ __forceinline__ uint32_t mbar_try4(uint32_t b0, uint32_t p0, uint32_t e0, uint32_t b1, uint32_t p1, uint32_t e1,
+                                              uint32_t b2, uint32_t p2, uint32_t e2, uint32_t b3, uint32_t p3, uint32_t e3) {
   uint32_t done;
   asm volatile(
-      "{\n\t.reg .pred q0, q1, q2, q3, q4, r0, r1, r2, r3, r4;\n\t"
-      "setp.ne.b32 q0, %3, 0;\n\tsetp.ne.b32 q1, %6, 0;\n\tsetp.ne.b32 q2, %9, 0;\n\t"
-      "setp.ne.b32 q3, %12, 0;\n\tsetp.ne.b32 q4, %15, 0;\n\t"
-      "setp.eq.b32 r0, 0, 0;\n\tsetp.eq.b32 r1, 0, 0;\n\tsetp.eq.b32 r2, 0, 0;\n\t"
-      "setp.eq.b32 r3, 0, 0;\n\tsetp.eq.b32 r4, 0, 0;\n\t"
+      "{\n\t.reg .pred q0, q1, q2, q3, r0, r1, r2, r3;\n\t"
+      "setp.ne.b32 q0, %3, 0;\n\tsetp.ne.b32 q1, %6, 0;\n\tsetp.ne.b32 q2, %9, 0;\n\tsetp.ne.b32 q3, %12, 0;\n\t"
+      "setp.eq.b32 r0, 0, 0;\n\tsetp.eq.b32 r1, 0, 0;\n\tsetp.eq.b32 r2, 0, 0;\n\tsetp.eq.b32 r3, 0, 0;\n\t"
       "@q0 mbarrier.try_wait.parity.shared::cta.b64 r0, [%1], %2;\n\t"
       "@q1 mbarrier.try_wait.parity.shared::cta.b64 r1, [%4], %5;\n\t"
       "@q2 mbarrier.try_wait.parity.shared::cta.b64 r2, [%7], %8;\n\t"
       "@q3 mbarrier.try_wait.parity.shared::cta.b64 r3, [%10], %11;\n\t"
-      "@q4 mbarrier.try_wait.parity.shared::cta.b64 r4, [%13], %14;\n\t"
-      "and.pred r0, r0, r1;\n\tand.pred r2, r2, r3;\n\tand.pred r0, r0, r4;\n\tand.pred r0, r0, r2;\n\t"
+      "and.pred r0, r0, r1;\n\tand.pred r2, r2, r3;\n\tand.pred r0, r0, r2;\n\t"
       "selp.u32 %0, 1, 0, r0;\n\t}"
       : "=r"(done)
       : "r"(b0), "r"(p0), "r"((uint32_t)e0), "r"(b1), "r"(p1), "r"((uint32_t)e1), "r"(b2), "r"(p2), "r"((uint32_t)e2),
-        "r"(b3), "r"(p3), "r"((uint32_t)e3), "r"(b4), "r"(p4), "r"((uint32_t)e4)
+        "r"(b3), "r"(p3), "r"((uint32_t)e3)
       : "memory");
   return done;
 }
@@ -359,6 +359,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       mbar_init(bar(Smem::q_empty, i), 1);
       mbar_init(bar(Smem::s_full, i), 1);
       mbar_init(bar(Smem::p_ready, i), 4);   // one arrival per softmax warp
+      mbar_init(bar(Smem::p_early, i), 4);   // likewise
       mbar_init(bar(Smem::o_full, i), 1);
       mbar_init(bar(Smem::o_free, i), 4);    // one arrival per softmax warp
     }
@@ -476,6 +477,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             pk[c / 2 + 1] = pack_bf16(p1.x, p1.y);
           }
           tmem_st16(s_addr + g * 16, pk);
+          if (g == BLK / 32 - 2) {
+            // all but the last 32 key columns of P are stored: their share of P V may start
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(Smem::p_early, X));
+          }
         }
         l_run += (sum_a.x + sum_a.y) + (sum_b.x + sum_b.y);
         tmem_st_wait();
@@ -633,10 +641,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       }
     } else if (warp == 9) {
       // ============================== MMA scheduler ==============================
-      // Decides what the tensor core does next and checks that it can be done (P ready, K / V and
-      // Q landed, O drained); the MMAs themselves are issued by warp 11 from a small command ring.
-      // tcgen05.mma issue blocks while the short tensor queue is full, so a warp that both waits on
-      // barriers and issues leaves the tensor core idle during its own book-keeping.
+      // Decides what the tensor core does next and checks ahead of time that it can be done (K / V
+      // and Q landed, O drained); the MMAs themselves are issued by warp 11 from a small command
+      // ring.  The scheduler runs ahead of the issuer, so that a visit's command is already waiting
+      // when the slot's softmax warps publish P: the issuer alone waits for P, and the path from
+      // "P stored" to "P V issued" is one barrier wake-up instead of a chain of book-keeping.
       Ctx ctx{abort_flag, a.status, kRoleMma};
       volatile uint32_t* cmd_word = (volatile uint32_t*)(smem_gen + Smem::cmd_word);
       uint32_t ci = 0, cpar = 0;  // next command slot and its phase
@@ -657,13 +666,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const bool need_o = do_pv && s.pend_first, need_q = do_qk && s.e == 0;
         const bool last = do_qk && s.e == s.cur.n - 1;
         const uint32_t all_done =
-            mbar_try5(bar(Smem::p_ready, X), s.p_par, do_pv, bar(Smem::kv_full, slot_v), par_v, do_pv,
-                      bar(Smem::o_free, X), s.o_par ^ 1, need_o, bar(Smem::kv_full, slot_k), par_k, do_qk,
-                      bar(Smem::q_full, X), s.q_par, need_q);
+            mbar_try4(bar(Smem::kv_full, slot_v), par_v, do_pv, bar(Smem::o_free, X), s.o_par ^ 1, need_o,
+                      bar(Smem::kv_full, slot_k), par_k, do_qk, bar(Smem::q_full, X), s.q_par, need_q);
         if (!__all_sync(0xffffffffu, all_done != 0)) {
           bool ok = true;
-          if (do_pv) ok = mbar_wait(bar(Smem::p_ready, X), s.p_par, ctx, kBarPReady) &&
-                          mbar_wait(bar(Smem::kv_full, slot_v), par_v, ctx, kBarKvFull);
+          if (do_pv) ok = mbar_wait(bar(Smem::kv_full, slot_v), par_v, ctx, kBarKvFull);
           if (ok && need_o) ok = mbar_wait(bar(Smem::o_free, X), s.o_par ^ 1, ctx, kBarOFree);
           if (ok && do_qk) ok = mbar_wait(bar(Smem::kv_full, slot_k), par_k, ctx, kBarKvFull);
           if (ok && need_q) ok = mbar_wait(bar(Smem::q_full, X), s.q_par, ctx, kBarQFull);
@@ -674,7 +681,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (lane == 0) {
           cmd_word[ci] = (do_pv ? kCmdPv : 0u) | (do_qk ? kCmdQk : 0u) | (s.pend_first ? kCmdPvFirst : 0u) |
                          (s.pend_last ? kCmdPvLast : 0u) | (last ? kCmdQkLast : 0u) | (X ? kCmdSlot1 : 0u) |
-                         (slot_v << 8) | (slot_k << 12);
+                         (s.p_par ? kCmdPPar : 0u) | (slot_v << 8) | (slot_k << 12);
           mbar_arrive(bar(Smem::cmd_full, ci));  // release: the word and everything observed above
         }
         __syncwarp();
@@ -724,6 +731,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       volatile uint32_t* cmd_word = (volatile uint32_t*)(smem_gen + Smem::cmd_word);
       uint32_t ci = 0, cpar = 0;
       bool ok = true;
+      const bool leader = elect_one();  // one lane issues every MMA and commit (a commit covers its own thread's MMAs)
       for (;;) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(Smem::cmd_full, ci), cpar, ctx, kBarCmdFull));
         if (!ok) break;
@@ -736,15 +744,38 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t slot_v = (cmd >> 8) & 15u, slot_k = (cmd >> 12) & 15u;
         const uint32_t s_tmem = tmem_base + X * 128;
         const uint32_t o_tmem = tmem_base + kOCol + X * 128;
-        tc_fence_after();
-        if (elect_one()) {
-          if (cmd & kCmdPv) {
-            const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
+        constexpr int kEarlySteps = (BLK / 32 - 1) * 2;  // 16-key steps of P V covered by p_early
+        const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
+        const uint32_t p_par = (cmd & kCmdPPar) ? 1u : 0u;
+        if (cmd & kCmdPv) {
+          // The one condition the scheduler leaves open: the slot's softmax warps have stored P.
+          // P V starts on the leading key columns while the softmax still works on the last 32.
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(Smem::p_early, X), p_par, ctx, kBarPEarly));
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
             const uint32_t first = (cmd & kCmdPvFirst) ? 1u : 0u;
-#pragma unroll
-            for (int k = 0; k < BLK / 16; ++k) {
-              const uint64_t db = smem_desc(v_addr + k * 2048, kHalfBytes, 1024);
-              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, (!first || k > 0) ? 1u : 0u);
+            uint64_t db = smem_desc(v_addr, kHalfBytes, 1024);
+            uint32_t acc = first ^ 1u;
+#pragma unroll 1
+            for (int k = 0; k < kEarlySteps; ++k) {  // rolled: the issuing loop stays within a few instruction-cache lines
+              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, acc);
+              db += 2048 >> 4;
+              acc = 1u;
+            }
+          }
+          __syncwarp();
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(Smem::p_ready, X), p_par, ctx, kBarPReady));
+          if (!ok) break;
+        }
+        tc_fence_after();
+        if (leader) {
+          if (cmd & kCmdPv) {
+            uint64_t db = smem_desc(v_addr + kEarlySteps * 2048, kHalfBytes, 1024);
+#pragma unroll 1
+            for (int k = kEarlySteps; k < BLK / 16; ++k) {
+              mma_ts(o_tmem, s_tmem + k * 8, db, kIdescPV, 1u);
+              db += 2048 >> 4;
             }
             tc_commit(bar(Smem::kv_empty, slot_v));
             if (cmd & kCmdPvLast) tc_commit(bar(Smem::o_full, X));
@@ -752,11 +783,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           if (cmd & kCmdQk) {
             const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
             const uint32_t k_addr = smem_base + Smem::kv + slot_k * kSlotBytes;
-#pragma unroll
+            uint64_t da = smem_desc(q_addr, 16, 1024);
+            uint64_t db = smem_desc(k_addr, 16, 1024);
+            uint32_t acc = 0u;
+#pragma unroll 1
             for (int k = 0; k < kHeadDim / 16; ++k) {
-              const uint64_t da = smem_desc(q_addr + (k >> 2) * (kTileM * 128) + (k & 3) * 32, 16, 1024);
-              const uint64_t db = smem_desc(k_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
-              mma_ss(s_tmem, da, db, kIdescS, k > 0 ? 1u : 0u);
+              mma_ss(s_tmem, da, db, kIdescS, acc);
+              acc = 1u;
+              // 16 columns = 32 bytes on; after four steps the next 64-column half of the tile
+              da += (k == 3) ? (uint64_t)((kTileM * 128 - 96) >> 4) : (uint64_t)(32 >> 4);
+              db += (k == 3) ? (uint64_t)((kHalfBytes - 96) >> 4) : (uint64_t)(32 >> 4);
             }
             tc_commit(bar(Smem::kv_empty, slot_k));
             tc_commit(bar(Smem::s_full, X));
