@@ -77,7 +77,7 @@ typedef struct stem_plan stem_plan; /* opaque; owns small host and device tables
 
 /* Sizes a caller needs to allocate buffers for a plan. */
 typedef struct {
-  size_t workspace_bytes;       /* scratch the hot calls need (pooled tensors, lists, status)      */
+  size_t workspace_bytes;       /* scratch the hot calls need (pooled tensors, metric, lists, status) */
   int32_t total_tokens;         /* T                                                               */
   int32_t total_q_blocks;       /* R_tot                                                           */
   int32_t k_max;                /* longest index list = max_r k_eff(r)                             */
@@ -148,13 +148,14 @@ int stem_score_static(const stem_plan* plan, const void* Q, const void* K, const
  *   For every (head, row): keeps the forced blocks {0..stem-1} and {r-local+1..r}, then adds the
  *   causal blocks of largest metric until the row holds k_eff(r) blocks.  Order: metric
  *   descending, block id ascending on equal metric, -0 == +0, NaN below every number.
- *   Reads M (layout above) if M != NULL, else recomputes metric rows from the pooled tensors a
- *   preceding stem_score left in the same workspace.  Writes sel_idx / sel_cnt. */
+ *   Reads M (layout above) if M != NULL, else recomputes the metric (into the workspace) from the
+ *   pooled tensors a preceding stem_score left in the same workspace.  Writes sel_idx / sel_cnt. */
 int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t* sel_cnt, void* workspace,
                 size_t workspace_bytes, void* stream);
 
 /* Alg. 1 steps 1-3c in one call: block-wise representations, Output-Aware Metric (Eq. 7), Token
- * Position-Decay budget (Eq. 3) and top-k selection, without materialising M.
+ * Position-Decay budget (Eq. 3) and top-k selection; the metric is kept in the workspace
+ *   (fp32 [num_q_heads, metric_elems], part of workspace_bytes), never handed to the caller.
  *   Same results as stem_score(M = NULL) followed by stem_select(M = NULL).
  *   Writes sel_idx / sel_cnt; leaves the pooled tensors in the workspace. */
 int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const void* V, int32_t* sel_idx,

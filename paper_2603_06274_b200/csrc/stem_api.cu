@@ -181,6 +181,18 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     p.n_sel_tiles = (int32_t)t.size();
   }
 
+  // Tiles of the metric GEMM: the 128 x 128 tiles of every sequence's causal triangle, long rows first.
+  std::vector<int32_t> gemm_tiles;
+  {
+    int max_t = 0;
+    for (int b = 0; b < batch; ++b) max_t = std::max(max_t, (seq_nblk[b] + 127) / 128);
+    for (int ti = max_t - 1; ti >= 0; --ti)
+      for (int b = 0; b < batch; ++b)
+        if (ti < (seq_nblk[b] + 127) / 128)
+          for (int tj = 0; tj <= ti; ++tj) { gemm_tiles.push_back(b); gemm_tiles.push_back(ti); gemm_tiles.push_back(tj); }
+    p.n_gemm_tiles = (int32_t)(gemm_tiles.size() / 3);
+  }
+
   // Attention work order: kv-head-major so that the K/V of one kv head stay hot in L2; inside a
   // kv head, rows by descending list length (longest first), the g heads of a row together.
   std::vector<int32_t> work_sparse, work_dense;
@@ -206,6 +218,9 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     p.ws.qbar = off;   off = align_up(off + (size_t)Hq * p.R_tot * kHeadDim * 4, 256);
     p.ws.kbar = off;   off = align_up(off + (size_t)Hkv * kHeadDim * p.kt_width * 4, 256);
     p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
+    p.ws.qsplit = off; off = align_up(off + (size_t)3 * Hq * p.R_tot * kHeadDim * 2, 256);
+    p.ws.ksplit = off; off = align_up(off + (size_t)3 * Hkv * p.R_tot * kHeadDim * 2, 256);
+    p.ws.metric = off; off = align_up(off + (size_t)Hq * (size_t)p.m_tot * 4, 256);
     p.ws.sel_idx = off; off = align_up(off + (size_t)Hq * p.R_tot * p.k_max * 4, 256);
     p.ws.sel_cnt = off; off = align_up(off + (size_t)Hq * p.R_tot * 4, 256);
     p.ws.total = off;
@@ -224,7 +239,8 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
                o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
                o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off),
                o_seq_kt_off = push(blob, seq_kt_off),
-               o_tiles = push(blob, tiles), o_ws = push(blob, work_sparse), o_wd = push(blob, work_dense);
+               o_tiles = push(blob, tiles), o_gt = push(blob, gemm_tiles), o_ws = push(blob, work_sparse),
+               o_wd = push(blob, work_dense);
   if (cudaMalloc(&p.d_blob, blob.size()) != cudaSuccess ||
       cudaMemcpy(p.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
     cudaGetLastError();
@@ -245,6 +261,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
   p.rows.seq_kt_off = (const int32_t*)(d + o_seq_kt_off);
   p.d_sel_tiles = (const int32_t*)(d + o_tiles);
+  p.d_gemm_tiles = (const int32_t*)(d + o_gt);
   p.d_work_sparse = (const int32_t*)(d + o_ws);
   p.d_work_dense = (const int32_t*)(d + o_wd);
   *out = sp;
@@ -308,16 +325,24 @@ static int check_ws(const Plan& p, const void* ws, size_t bytes) {
 
 static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
 
-// Alg. 1 steps 1-3c: pooling, then scoring + selection of every tile, on one stream.
-// (Two ways of overlapping the HBM-bound pooling with the FMA-bound scoring were measured and
-// dropped: phases on two streams lose more to cross-stream event waits than they gain, and one
-// persistent kernel with a shared ticket list leaves too few warps per SM to stream HBM.)
-static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar,
-                                float* mv, int32_t* idx, int32_t* cnt, cudaStream_t s) {
-  int rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+// Alg. 1 steps 1-3c on one stream: pooling (one pass over Q, K, V; also emits the pooled vectors as
+// bf16 parts), the metric of every causal block on the tensor cores into the workspace, and the
+// row-wise selection from it.
+// (Two ways of overlapping the HBM-bound pooling with the scoring were measured and dropped: phases
+// on two streams lose more to cross-stream event waits than they gain, and one persistent kernel
+// with a shared ticket list leaves too few warps per SM to stream HBM.)
+static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, uint8_t* w, int32_t* idx,
+                                int32_t* cnt, cudaStream_t s) {
+  float* mv = (float*)(w + p.ws.mv);
+  float* M = (float*)(w + p.ws.metric);
+  int rc = cuda_rc(launch_pool(p, Q, K, V, (float*)(w + p.ws.qbar), (float*)(w + p.ws.kbar), mv, w + p.ws.qsplit,
+                               w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_score_select(p, kFromPooled | kSelect, qbar, kbar, mv, nullptr, nullptr, idx, cnt, s));
+  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, (int32_t*)(w + p.ws.status), s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  rc = cuda_rc(launch_select_rows(p, M, idx, cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }
@@ -335,11 +360,11 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   float* qbar = (float*)(w + p.ws.qbar);
   float* kbar = (float*)(w + p.ws.kbar);
   float* mv = (float*)(w + p.ws.mv);
-  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   if (M) {
-    rc = cuda_rc(launch_score_select(p, kFromPooled | kWriteMetric, qbar, kbar, mv, nullptr, M, nullptr, nullptr, s));
+    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, (int32_t*)(w + p.ws.status), s));
     if (rc != STEM_OK) return rc;
     p.last_launches++;
   }
@@ -355,9 +380,17 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
   p.last_launches = 0;
-  const int mode = (M ? kFromMetric : kFromPooled) | kSelect;
-  rc = cuda_rc(launch_score_select(p, mode, (const float*)(w + p.ws.qbar), (const float*)(w + p.ws.kbar),
-                                   (const float*)(w + p.ws.mv), M, nullptr, sel_idx, sel_cnt, (cudaStream_t)stream));
+  cudaStream_t s = (cudaStream_t)stream;
+  if (!M) {
+    // recompute the metric from the pooled vectors a previous stem_score left in the workspace
+    float* Mw = (float*)(w + p.ws.metric);
+    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, (const float*)(w + p.ws.mv), Mw,
+                                    (int32_t*)(w + p.ws.status), s));
+    if (rc != STEM_OK) return rc;
+    p.last_launches++;
+    M = Mw;
+  }
+  rc = cuda_rc(launch_select_rows(p, M, sel_idx, sel_cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }
@@ -372,8 +405,7 @@ int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
   p.last_launches = 0;
-  return enqueue_score_select(p, Q, K, V, (float*)(w + p.ws.qbar), (float*)(w + p.ws.kbar), (float*)(w + p.ws.mv),
-                              sel_idx, sel_cnt, (cudaStream_t)stream);
+  return enqueue_score_select(p, Q, K, V, w, sel_idx, sel_cnt, (cudaStream_t)stream);
 }
 
 int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, const int32_t* sel_idx,
@@ -401,13 +433,10 @@ int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
   cudaStream_t s = (cudaStream_t)stream;
-  float* qbar = (float*)(w + p.ws.qbar);
-  float* kbar = (float*)(w + p.ws.kbar);
-  float* mv = (float*)(w + p.ws.mv);
   int32_t* idx = sel_idx ? sel_idx : (int32_t*)(w + p.ws.sel_idx);
   int32_t* cnt = sel_cnt ? sel_cnt : (int32_t*)(w + p.ws.sel_cnt);
   p.last_launches = 0;
-  rc = enqueue_score_select(p, Q, K, V, qbar, kbar, mv, idx, cnt, s);
+  rc = enqueue_score_select(p, Q, K, V, w, idx, cnt, s);
   if (rc != STEM_OK) return rc;
   rc = cuda_rc(launch_sparse_attention(p, Q, K, V, idx, cnt, O, lse, (int32_t*)(w + p.ws.status), s));
   if (rc != STEM_OK) return rc;
@@ -424,7 +453,8 @@ int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* de
   if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   if (cudaMemcpy(words, w, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   if (detail) std::memcpy(detail, words, 4 * sizeof(int32_t));
-  if (words[0] != 0) {
+  if (words[0] != 0 || words[4] != 0) {
+    if (detail && words[0] == 0) std::memcpy(detail, words + 4, 4 * sizeof(int32_t));  // the metric kernel's words
     cudaMemset(w, 0, sizeof(words));
     return STEM_ERR_DEVICE_TIMEOUT;
   }

@@ -13,7 +13,8 @@ namespace stem {
 constexpr int kHeadDim = 128;
 
 // Status words at the start of the workspace (int32 each).
-//   [0] code (0 = ok, 1 = a bounded wait gave up)   [1] CTA index   [2] role   [3] barrier id
+//   [0] code (0 = ok, 1 = a bounded wait of the attention kernel gave up)   [1] CTA index   [2] role   [3] barrier id
+//   [4] code (2 = a bounded wait of the metric kernel gave up)   [5] tile   [6] head
 constexpr int kStatusWords = 8;
 
 // Device-side row tables, built once per plan.
@@ -37,6 +38,9 @@ struct WorkspaceLayout {
   size_t qbar = 0;     // fp32 [H_q, R_tot, d]
   size_t kbar = 0;     // fp32 [H_kv, d, kt_width]: Kbar transposed, block index contiguous
   size_t mv = 0;       // fp32 [H_kv, R_tot]
+  size_t qsplit = 0;   // bf16 [3, H_q, R_tot, d]: Qbar as hi + mid + lo parts
+  size_t ksplit = 0;   // bf16 [3, H_kv, R_tot, d]: Kbar likewise (row = global block row)
+  size_t metric = 0;   // fp32 [H_q, m_tot]: M of the fused path
   size_t sel_idx = 0;  // int32 [H_q, R_tot, k_max]
   size_t sel_cnt = 0;  // int32 [H_q, R_tot]
   size_t total = 0;
@@ -61,6 +65,8 @@ struct Plan {
   int32_t n_sel_tiles = 0;
   int32_t sel_rows_per_tile = 0;         // rows of one tile (all heads of a kv group ride together)
   int32_t sel_nq = 0;                    // pooled query vectors per tile
+  const int32_t* d_gemm_tiles = nullptr;  // [n_gemm_tiles][3] (sequence, row tile, column tile) of the metric GEMM
+  int32_t n_gemm_tiles = 0;
   const int32_t* d_work_sparse = nullptr;  // [n_items][2] (head, global row), attention work order
   const int32_t* d_work_dense = nullptr;
   int32_t n_items = 0;
@@ -71,8 +77,13 @@ struct Plan {
 
 // Kernel launchers (each returns the cudaError_t of the launch).
 // qbar: [H_q, R_tot, d]; kbar_t: [H_kv, d, kt_width] (transposed for the scoring GEMM); mv: [H_kv, R_tot].
+// qsplit / ksplit (optional, both or neither): bf16 [3, H, R_tot, d], the pooled vectors as hi + mid + lo parts.
 cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t,
-                        float* mv, cudaStream_t s);
+                        float* mv, void* qsplit, void* ksplit, cudaStream_t s);
+
+// Metric of every causal block (layout of stem_score's M) from the split pooled vectors, on the tensor cores.
+cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
+                               int32_t* status, cudaStream_t s);
 
 // Shared-memory needs of the score/select kernel, for sizing its tiles at plan creation.
 size_t score_select_list_bytes(int k_max);   // per pooled query vector
@@ -84,6 +95,10 @@ enum : int { kFromPooled = 1, kFromMetric = 2, kWriteMetric = 4, kSelect = 8 };
 cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar_t, const float* mv,
                                 const float* M_in, float* M_out, int32_t* sel_idx, int32_t* sel_cnt,
                                 cudaStream_t s);
+
+// Selection from a stored metric (layout of stem_score's M), one warp per (head, row).
+int row_select_max_blocks();  // largest supported N_blk of a sequence
+cudaError_t launch_select_rows(const Plan& p, const float* M, int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
 
 cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
                                     const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,

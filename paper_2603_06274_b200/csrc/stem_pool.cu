@@ -37,7 +37,8 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
                                                    const __nv_bfloat16* __restrict__ V, int64_t q_st, int64_t q_sh,
                                                    int64_t kv_st, int64_t kv_sh, int Hq, int Hkv, int R_tot, int kt_width,
                                                    RowTables rows, float* __restrict__ qbar, float* __restrict__ kbar_t,
-                                                   float* __restrict__ mv) {
+                                                   float* __restrict__ mv, __nv_bfloat16* __restrict__ qsplit,
+                                                   __nv_bfloat16* __restrict__ ksplit) {
   constexpr int kTokPerWarp = kBlock / 4;
   constexpr int kSteps = kTokPerWarp / 2;
   const int slots = Hq + 2 * Hkv;
@@ -86,6 +87,20 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
     const int c = threadIdx.x;
     const float sum = (red[0][c] + red[1][c]) + (red[2][c] + red[3][c]);
     const float mean = sum / (float)ntok;
+    if (qsplit != nullptr) {
+      // mean = hi + mid + lo, each part the bf16 rounding of what the previous ones leave (the tensor-core
+      // metric kernel multiplies these parts); row = global block row for both tensors
+      const __nv_bfloat16 hi = __float2bfloat16_rn(mean);
+      const float r1 = mean - __bfloat162float(hi);
+      const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+      const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+      __nv_bfloat16* dst = kind == 0 ? qsplit : ksplit;
+      const int64_t plane = (int64_t)(kind == 0 ? Hq : Hkv) * R_tot * kHeadDim;
+      const int64_t at = ((int64_t)h * R_tot + R) * kHeadDim + c;
+      dst[at] = hi;
+      dst[at + plane] = mid;
+      dst[at + 2 * plane] = lo;
+    }
     if (kind == 0) {
       qbar[((int64_t)h * R_tot + R) * kHeadDim + c] = mean;
     } else {
@@ -121,7 +136,7 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
 }  // namespace
 
 cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t, float* mv,
-                        cudaStream_t s) {
+                        void* qsplit, void* ksplit, cudaStream_t s) {
   const int slots = p.cfg.num_q_heads + 2 * p.cfg.num_kv_heads;
   const dim3 grid((unsigned)((int64_t)p.R_tot * slots));
   auto q = (const __nv_bfloat16*)Q;
@@ -130,11 +145,11 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
   if (p.cfg.block == 128)
     pool_kernel<128><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
                                           p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
-                                          p.rows, qbar, kbar_t, mv);
+                                          p.rows, qbar, kbar_t, mv, (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
   else
     pool_kernel<64><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
                                          p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
-                                         p.rows, qbar, kbar_t, mv);
+                                         p.rows, qbar, kbar_t, mv, (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
   return cudaGetLastError();
 }
 

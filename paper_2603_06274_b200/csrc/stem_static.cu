@@ -63,7 +63,7 @@ extern "C" int stem_score_static(const stem_plan* plan, const void* Q, const voi
   p.last_launches = 0;
   // The pooling kernel writes every element of qbar / kbar / mv that the metric kernel reads, so
   // whatever an earlier call left in the array is never observed.
-  if (launch_pool(p, Q, K, V, qbar, kbar, mv, s) != cudaSuccess) return STEM_ERR_CUDA;
+  if (launch_pool(p, Q, K, V, qbar, kbar, mv, nullptr, nullptr, s) != cudaSuccess) return STEM_ERR_CUDA;
   p.last_launches++;
   if (launch_score_select(p, kFromPooled | kWriteMetric, qbar, kbar, mv, nullptr, M, nullptr, nullptr, s) != cudaSuccess)
     return STEM_ERR_CUDA;
