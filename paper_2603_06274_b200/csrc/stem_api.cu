@@ -215,8 +215,6 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   {
     size_t off = 0;
     p.ws.status = off; off = align_up(off + kStatusWords * 4, 256);
-    p.ws.qbar = off;   off = align_up(off + (size_t)Hq * p.R_tot * kHeadDim * 4, 256);
-    p.ws.kbar = off;   off = align_up(off + (size_t)Hkv * kHeadDim * p.kt_width * 4, 256);
     p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
     p.ws.qsplit = off; off = align_up(off + (size_t)3 * Hq * p.R_tot * kHeadDim * 2, 256);
     p.ws.ksplit = off; off = align_up(off + (size_t)3 * Hkv * p.R_tot * kHeadDim * 2, 256);
@@ -335,8 +333,7 @@ static int enqueue_score_select(const Plan& p, const void* Q, const void* K, con
                                 int32_t* cnt, cudaStream_t s) {
   float* mv = (float*)(w + p.ws.mv);
   float* M = (float*)(w + p.ws.metric);
-  int rc = cuda_rc(launch_pool(p, Q, K, V, (float*)(w + p.ws.qbar), (float*)(w + p.ws.kbar), mv, w + p.ws.qsplit,
-                               w + p.ws.ksplit, s));
+  int rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, (int32_t*)(w + p.ws.status), s));
@@ -357,10 +354,8 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   uint8_t* w = (uint8_t*)ws;
   cudaStream_t s = (cudaStream_t)stream;
   p.last_launches = 0;
-  float* qbar = (float*)(w + p.ws.qbar);
-  float* kbar = (float*)(w + p.ws.kbar);
   float* mv = (float*)(w + p.ws.mv);
-  rc = cuda_rc(launch_pool(p, Q, K, V, qbar, kbar, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   if (M) {

@@ -35,8 +35,6 @@ struct RowTables {
 // Where things live inside the caller's workspace (byte offsets, 256-aligned).
 struct WorkspaceLayout {
   size_t status = 0;
-  size_t qbar = 0;     // fp32 [H_q, R_tot, d]
-  size_t kbar = 0;     // fp32 [H_kv, d, kt_width]: Kbar transposed, block index contiguous
   size_t mv = 0;       // fp32 [H_kv, R_tot]
   size_t qsplit = 0;   // bf16 [3, H_q, R_tot, d]: Qbar as hi + mid + lo parts
   size_t ksplit = 0;   // bf16 [3, H_kv, R_tot, d]: Kbar likewise (row = global block row)
@@ -77,7 +75,8 @@ struct Plan {
 
 // Kernel launchers (each returns the cudaError_t of the launch).
 // qbar: [H_q, R_tot, d]; kbar_t: [H_kv, d, kt_width] (transposed for the scoring GEMM); mv: [H_kv, R_tot].
-// qsplit / ksplit (optional, both or neither): bf16 [3, H, R_tot, d], the pooled vectors as hi + mid + lo parts.
+// qbar / kbar_t (optional, fp32) and qsplit / ksplit (optional, both or neither: bf16 [3, H, R_tot, d], the pooled
+// vectors as hi + mid + lo parts) are two forms of the same pooled vectors; a caller asks for the one it reads.
 cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t,
                         float* mv, void* qsplit, void* ksplit, cudaStream_t s);
 

@@ -11,8 +11,9 @@
 // terms are below 2^-24 of the leading one.  A pooled value that is not finite makes its row or
 // column of M NaN (which ranks below every number).
 //
-// One CTA per (128 x 128 tile of one sequence's causal triangle, query head): TMA brings the
-// 3 + 3 operand tiles (K-major, 128-byte swizzle), one thread issues the 48 MMAs, the four warps
+// One CTA per (128 x 128 tile of one sequence's causal triangle, query head), two CTAs per SM: TMA
+// brings the 3 + 3 operand parts (K-major, 128-byte swizzle) one half of the head dimension at a
+// time, one thread issues the 2 x 24 MMAs, the four warps
 // read the accumulator (one row per thread), apply scale and bias, turn the tile through shared
 // memory and write the causal part of it with coalesced stores.  Waits are bounded.
 #include <cuda.h>
@@ -26,14 +27,14 @@ namespace {
 
 constexpr int kThreads = 128;
 constexpr int kTile = 128;
-constexpr int kOpBytes = kTile * kHeadDim * 2;       // one operand tile (bf16): 32 KB
-constexpr int kHalf = kTile * 128;                   // its 64-column half
-constexpr int kSmemOps = 6 * kOpBytes;               // A hi/mid/lo, B hi/mid/lo
-constexpr int kSmemBias = kSmemOps;                  // 128 floats
-constexpr int kSmemBars = kSmemBias + kTile * 4;     // full, done
-constexpr int kSmemTmem = kSmemBars + 16;
+constexpr int kPartBytes = kTile * 128;               // one operand part, one 64-column half of d (bf16): 16 KB
+constexpr int kSmemOps = 6 * kPartBytes;              // A hi/mid/lo, B hi/mid/lo (reused for both halves of d)
+constexpr int kSmemBias = kSmemOps;                   // 128 floats
+constexpr int kSmemBars = kSmemBias + kTile * 4;      // full, half_done, done
+constexpr int kSmemTmem = kSmemBars + 32;
 constexpr int kSmemTotal = kSmemTmem + 16;
-constexpr int kSmemBytes = kSmemTotal + 1024;        // slack for manual 1024-byte alignment
+constexpr int kSmemBytes = kSmemTotal + 1024;         // slack for manual 1024-byte alignment; two CTAs per SM
+static_assert(kTile * kTile * 4 <= kSmemOps, "the output tile is staged over the operand tiles");
 constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
 
 __device__ __forceinline__ uint64_t globaltimer() {
@@ -138,13 +139,13 @@ struct GemmArgs {
   float beta, scale;
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const GemmArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - (uint32_t)__cvta_generic_to_shared(smem_raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t bar_full = smem_base + kSmemBars, bar_done = bar_full + 8;
+  const uint32_t bar_full = smem_base + kSmemBars, bar_half = bar_full + 8, bar_done = bar_full + 16;
   float* bias = (float*)(smem_gen + kSmemBias);
 
   const int seq = a.tiles[3 * blockIdx.x], ti = a.tiles[3 * blockIdx.x + 1], tj = a.tiles[3 * blockIdx.x + 2];
@@ -155,6 +156,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
   if (threadIdx.x == 0) {
     mbar_init(bar_full, 1);
+    mbar_init(bar_half, 1);
     mbar_init(bar_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -175,37 +177,40 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
   bool ok = true;
   if (warp == 0) {
+    // The head dimension goes through shared memory in two halves of 64 columns (six 16 KB parts
+    // each), so that two CTAs fit on an SM and one's copies overlap the other's MMAs and epilogue.
     const bool leader = elect_one();
-    if (leader) {
-      mbar_expect_tx(bar_full, kSmemOps);
+    // parts of A x parts of B, smallest products first: (mid,mid) (hi,lo) (lo,hi) (hi,mid) (mid,hi) (hi,hi)
+    constexpr int kPairs[6][2] = {{1, 1}, {0, 2}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};
+    uint32_t acc = 0u;
+#pragma unroll 1
+    for (int half = 0; half < 2 && ok; ++half) {
+      if (half == 1) ok = __all_sync(0xffffffffu, mbar_wait(bar_half, 0, a.status));  // the first half's MMAs have read the parts
+      if (!ok) break;
+      if (leader) {
+        mbar_expect_tx(bar_full, kSmemOps);
 #pragma unroll
-      for (int s = 0; s < 3; ++s) {
-        tma_load_3d(smem_base + s * kOpBytes, &map_q, bar_full, 0, R0, s * a.Hq + h);
-        tma_load_3d(smem_base + s * kOpBytes + kHalf, &map_q, bar_full, 64, R0, s * a.Hq + h);
-        tma_load_3d(smem_base + (3 + s) * kOpBytes, &map_k, bar_full, 0, C0, s * a.Hkv + kvh);
-        tma_load_3d(smem_base + (3 + s) * kOpBytes + kHalf, &map_k, bar_full, 64, C0, s * a.Hkv + kvh);
+        for (int s = 0; s < 3; ++s) {
+          tma_load_3d(smem_base + s * kPartBytes, &map_q, bar_full, 64 * half, R0, s * a.Hq + h);
+          tma_load_3d(smem_base + (3 + s) * kPartBytes, &map_k, bar_full, 64 * half, C0, s * a.Hkv + kvh);
+        }
       }
-    }
-    __syncwarp();
-    ok = __all_sync(0xffffffffu, mbar_wait(bar_full, 0, a.status));
-    if (ok) {
+      __syncwarp();
+      ok = __all_sync(0xffffffffu, mbar_wait(bar_full, half, a.status));
+      if (!ok) break;
       tc_fence_after();
       if (leader) {
-        // parts of A x parts of B, smallest products first: (mid,mid) (hi,lo) (lo,hi) (hi,mid) (mid,hi) (hi,hi)
-        constexpr int kPairs[6][2] = {{1, 1}, {0, 2}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};
-        uint32_t acc = 0u;
 #pragma unroll
         for (int q = 0; q < 6; ++q) {
-          const uint32_t a_addr = smem_base + kPairs[q][0] * kOpBytes;
-          const uint32_t b_addr = smem_base + (3 + kPairs[q][1]) * kOpBytes;
+          const uint32_t a_addr = smem_base + kPairs[q][0] * kPartBytes;
+          const uint32_t b_addr = smem_base + (3 + kPairs[q][1]) * kPartBytes;
 #pragma unroll
-          for (int k = 0; k < kHeadDim / 16; ++k) {
-            const uint32_t off = (k >> 2) * kHalf + (k & 3) * 32;
-            mma_ss(tmem, smem_desc(a_addr + off), smem_desc(b_addr + off), kIdesc, acc);
+          for (int k = 0; k < 4; ++k) {
+            mma_ss(tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), kIdesc, acc);
             acc = 1u;
           }
         }
-        tc_commit(bar_done);
+        tc_commit(half == 0 ? bar_half : bar_done);
       }
       __syncwarp();
     }

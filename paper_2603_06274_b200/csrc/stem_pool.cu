@@ -102,8 +102,8 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
       dst[at + 2 * plane] = lo;
     }
     if (kind == 0) {
-      qbar[((int64_t)h * R_tot + R) * kHeadDim + c] = mean;
-    } else {
+      if (qbar != nullptr) qbar[((int64_t)h * R_tot + R) * kHeadDim + c] = mean;
+    } else if (kbar_t != nullptr) {
       // Kbar is stored transposed ([H_kv, d, kt_width], block index contiguous) for the scoring GEMM
       const int col = rows.seq_kt_off[rows.row_seq[R]] + rows.row_r[R];
       kbar_t[((int64_t)h * kHeadDim + c) * kt_width + col] = mean;

@@ -4,11 +4,15 @@
 // A row's forced blocks are its first `stem` and last `local` causal blocks; the candidates are the
 // causal blocks between them.  The row takes the need = k_eff(r) - #forced best candidates by
 // (metric descending, block id ascending), metric compared as an order-preserving 32-bit key with
-// -0 == +0 and NaN as -inf.  The warp holds the candidates' keys in registers (candidate c of the row
-// in lane c % 32, register c / 32), finds the need-th largest key by a most-significant-bit-first
-// radix descent, one warp-wide population count per varying key bit, and writes the selected block
-// ids in ascending order.  For the descent each lane keeps its 32 keys bit-transposed (word b holds
-// bit b of every key), so that one AND and one popc per lane count a bit over the whole row.
+// -0 == +0 and NaN as -inf.
+// The warp reads the row's metric with coalesced loads and turns it through shared memory so that
+// every lane holds a run of consecutive candidates (lane L the candidates L*c .. L*c + c - 1,
+// c = ceil(n_cand / 32)).  Each lane bit-transposes its keys (word b = bit b of every key of the
+// lane), and the need-th largest key is found by a most-significant-bit-first radix descent that
+// costs one AND + popc per lane and one warp reduction per varying key bit, and stops as soon as
+// the keys still undecided are exactly the ones still needed.  The selected ids come out in
+// ascending order by a warp prefix sum over the lanes' counts.  The kernel is bound by the integer
+// pipe, so the stages are written for few logic instructions (byte permutes in the transpose).
 #include <cuda_runtime.h>
 
 #include "stem_internal.h"
@@ -30,16 +34,28 @@ __device__ __forceinline__ uint32_t metric_key(float f) {
 // In-register transpose of a 32 x 32 bit matrix: afterwards bit t of w[b] is bit b of the old w[t].
 __device__ __forceinline__ void transpose32(uint32_t (&w)[32]) {
 #pragma unroll
-  for (int s = 0; s < 5; ++s) {
+  for (int k = 0; k < 16; ++k) {  // 16-bit halves: byte permutes
+    const uint32_t lo = __byte_perm(w[k], w[k + 16], 0x5410), hi = __byte_perm(w[k], w[k + 16], 0x7632);
+    w[k] = lo;
+    w[k + 16] = hi;
+  }
+#pragma unroll
+  for (int k = 0; k < 32; ++k) {  // bytes
+    if (k & 8) continue;
+    const uint32_t lo = __byte_perm(w[k], w[k + 8], 0x6240), hi = __byte_perm(w[k], w[k + 8], 0x7351);
+    w[k] = lo;
+    w[k + 8] = hi;
+  }
+#pragma unroll
+  for (int s = 2; s < 5; ++s) {
     const int j = 16 >> s;
-    const uint32_t m = s == 0 ? 0xffff0000u : s == 1 ? 0xff00ff00u : s == 2 ? 0xf0f0f0f0u : s == 3 ? 0xccccccccu : 0xaaaaaaaau;
+    const uint32_t mhi = s == 2 ? 0xf0f0f0f0u : s == 3 ? 0xccccccccu : 0xaaaaaaaau;
 #pragma unroll
     for (int k = 0; k < 32; ++k) {
       if (k & j) continue;
-      // swap the high-j-bit part of row k with the low-j-bit part of row k + j
-      const uint32_t t = ((w[k] >> j) ^ w[k + j]) & (m >> j);
-      w[k] ^= t << j;
-      w[k + j] ^= t;
+      const uint32_t x = w[k], y = w[k + j];
+      w[k] = (x & ~mhi) | ((y << j) & mhi);
+      w[k + j] = ((x >> j) & ~mhi) | (y & mhi);
     }
   }
 }
@@ -53,11 +69,26 @@ struct SelArgs {
   int Hq, R_tot, k_max, stem, local;
 };
 
+// The mask of the n lowest set bits of m.
+__device__ __forceinline__ uint32_t lowest_bits(uint32_t m, int n) {
+  uint32_t r = 0u;
+  while (n > 0 && m != 0u) {
+    const uint32_t b = m & (0u - m);
+    r |= b;
+    m ^= b;
+    --n;
+  }
+  return r;
+}
+
 // SETS = 32-key register sets per lane: rows of up to SETS * 1024 candidates.
 template <int SETS>
 __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kernel(const SelArgs a) {
-  const int lane = threadIdx.x & 31;
-  const int64_t item = (int64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  constexpr int kStride = 32 * SETS + 1;  // words of shared memory per lane (odd: conflict-free both ways)
+  extern __shared__ uint32_t stage_all[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* stage = stage_all + warp * 32 * kStride;
+  const int64_t item = (int64_t)blockIdx.x * (kThreads / 32) + warp;
   if (item >= (int64_t)a.Hq * a.R_tot) return;
   // rows in descending order so that the long rows of a launch start first
   const int h = (int)(item % a.Hq);
@@ -72,89 +103,112 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
   const int n_forced = i - n_cand;
   const int need = max(min(a.rows.row_keff[R] - n_forced, n_cand), 0);
   int32_t* out = a.sel_idx + ((int64_t)h * a.R_tot + R) * a.k_max;
-  const float* mrow = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq] + (int64_t)r * nb;
-  const uint32_t lt_mask = (1u << lane) - 1u;
+  const float* mrow = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq] + (int64_t)r * nb + c_lo;
+  const int per = (n_cand + 31) >> 5;  // candidates per lane
 
-  // ---- keys of the candidates (0 = no candidate; every real key is >= 1), then bit-transposed in place
-  uint32_t tw[SETS][32];
-  uint32_t act[SETS], gt[SETS];  // per key of this lane (bit t <-> register t): still in the descent / known > T
-  uint32_t vary = 0u;
-  const uint32_t key0 = n_cand > 0 ? metric_key(mrow[c_lo]) : 0u;
+  uint32_t sel[SETS];  // per key of this lane (bit t <-> its t-th candidate): selected
 #pragma unroll
-  for (int s = 0; s < SETS; ++s) {
-    act[s] = 0u;
-    gt[s] = 0u;
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-      const int j = c_lo + (s * 32 + t) * 32 + lane;
-      uint32_t kx = 0u;
-      if ((s * 32 + t) * 32 < n_cand && j < c_hi) {
-        kx = metric_key(mrow[j]);
-        act[s] |= 1u << t;
-        vary |= kx ^ key0;
-      }
-      tw[s][t] = kx;
+  for (int s = 0; s < SETS; ++s) sel[s] = 0u;
+
+  if (need > 0) {
+    // ---- keys: coalesced loads, through shared memory into runs of `per` consecutive candidates per lane
+    const uint32_t magic = ((1u << 20) + per - 1) / per;  // q / per == (q * magic) >> 20 for q < 2048
+    for (int q = lane; q < n_cand; q += 32) {
+      const uint32_t owner = ((uint32_t)q * magic) >> 20;
+      stage[owner * kStride + (q - owner * per)] = metric_key(mrow[q]);
     }
-    transpose32(tw[s]);
-  }
+    __syncwarp();
+    uint32_t tw[SETS][32];
+    uint32_t act[SETS], gt[SETS];  // still in the descent / known to be above the threshold
+    uint32_t vary = 0u;
+    const uint32_t key0 = stage[0];
+    const int mine = min(max(n_cand - lane * per, 0), per);  // candidates of this lane
+#pragma unroll
+    for (int s = 0; s < SETS; ++s) {
+      gt[s] = 0u;
+      const int cnt_s = min(max(mine - 32 * s, 0), 32);
+      act[s] = cnt_s >= 32 ? 0xffffffffu : ((1u << cnt_s) - 1u);
+#pragma unroll
+      for (int t = 0; t < 32; ++t) {
+        uint32_t kx = 0u;
+        if (32 * s + t < per) {  // warp-uniform
+          kx = stage[lane * kStride + 32 * s + t];
+          if (32 * s + t >= mine) kx = 0u;
+          else vary |= kx ^ key0;
+        }
+        tw[s][t] = kx;
+      }
+      transpose32(tw[s]);
+    }
 
-  // ---- threshold: the need-th largest key T; gt = keys above it, act = keys equal to it
-  int rem = 0;  // how many of the keys equal to T are taken (the first ones by block id)
-  if (need == 0) {
-#pragma unroll
-    for (int s = 0; s < SETS; ++s) act[s] = 0u;
-  } else if (need == n_cand) {
-#pragma unroll
-    for (int s = 0; s < SETS; ++s) { gt[s] = act[s]; act[s] = 0u; }
-  } else {
+    // ---- the need-th largest key by radix descent; gt = keys above it, act = keys still undecided.
+    // The descent stops deciding as soon as the undecided keys are exactly the ones still needed
+    // (at once when every candidate is needed); at the end the undecided keys are all equal.
     vary = __reduce_or_sync(0xffffffffu, vary);
-    int k = need;  // rank wanted among the keys still active
+    int k = need, na = n_cand;  // rank wanted among the undecided keys, number of undecided keys
 #pragma unroll
     for (int b = 31; b >= 0; --b) {
-      if (!((vary >> b) & 1u)) continue;  // warp-uniform: all candidates agree on this bit
-      int cnt = 0;
+      if (((vary >> b) & 1u) != 0u && k != na) {  // warp-uniform; a bit all candidates agree on decides nothing
+        int cnt = 0;
 #pragma unroll
-      for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
-      cnt = __reduce_add_sync(0xffffffffu, cnt);
-      if (cnt >= k) {
+        for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
+        cnt = __reduce_add_sync(0xffffffffu, cnt);
+        if (cnt >= k) {
+          na = cnt;
 #pragma unroll
-        for (int s = 0; s < SETS; ++s) act[s] &= tw[s][b];
-      } else {
-        k -= cnt;
+          for (int s = 0; s < SETS; ++s) act[s] &= tw[s][b];
+        } else {
+          k -= cnt;
+          na -= cnt;
 #pragma unroll
-        for (int s = 0; s < SETS; ++s) { gt[s] |= act[s] & tw[s][b]; act[s] &= ~tw[s][b]; }
+          for (int s = 0; s < SETS; ++s) { gt[s] |= act[s] & tw[s][b]; act[s] &= ~tw[s][b]; }
+        }
       }
     }
-    rem = k;
-  }
-  // Equal keys beyond the ones needed are the rare case; otherwise every key equal to T is taken.
-  int n_eq = 0;
+    const int rem = k;  // of the undecided keys the first `rem` by block id are taken
+    // ---- the equal keys that are taken: the first `rem` in lane-major order
+    int n_eq = 0;
 #pragma unroll
-  for (int s = 0; s < SETS; ++s) n_eq += __popc(act[s]);
-  n_eq = __reduce_add_sync(0xffffffffu, n_eq);
-  const bool ties = n_eq > rem;
+    for (int s = 0; s < SETS; ++s) n_eq += __popc(act[s]);
+    int before = n_eq;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, before, d);
+      if (lane >= d) before += v;
+    }
+    before -= n_eq;  // equal keys in lower lanes
+    int quota = min(max(rem - before, 0), n_eq);
+#pragma unroll
+    for (int s = 0; s < SETS; ++s) {
+      const int take = min(quota, __popc(act[s]));
+      sel[s] = gt[s] | (take == __popc(act[s]) ? act[s] : lowest_bits(act[s], take));
+      quota -= take;
+    }
+  }
 
   // ---- emission in ascending block order: stem blocks, selected candidates, local blocks
   for (int j = lane; j < n_stem; j += 32) out[j] = j;
-  int base = n_stem, eq_before = 0;
+  int n_sel = 0;
+#pragma unroll
+  for (int s = 0; s < SETS; ++s) n_sel += __popc(sel[s]);
+  int pos = n_sel;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, pos, d);
+    if (lane >= d) pos += v;
+  }
+  const int n_taken = __shfl_sync(0xffffffffu, pos, 31);  // == need
+  pos += n_stem - n_sel;
 #pragma unroll
   for (int s = 0; s < SETS; ++s) {
-    const uint32_t sel = ties ? gt[s] : (gt[s] | act[s]);
-#pragma unroll
-    for (int t = 0; t < 32; ++t) {
-      if ((s * 32 + t) * 32 >= n_cand) break;  // warp-uniform
-      bool take = (sel >> t) & 1u;
-      if (ties) {
-        const bool eq = (act[s] >> t) & 1u;
-        const uint32_t eqb = __ballot_sync(0xffffffffu, eq);
-        take = take || (eq && eq_before + __popc(eqb & lt_mask) < rem);
-        eq_before += __popc(eqb);
-      }
-      const uint32_t selb = __ballot_sync(0xffffffffu, take);
-      if (take) out[base + __popc(selb & lt_mask)] = c_lo + (s * 32 + t) * 32 + lane;
-      base += __popc(selb);
+    uint32_t m = sel[s];
+    while (m != 0u) {
+      const int t = __ffs((int)m) - 1;
+      m &= m - 1u;
+      out[pos++] = c_lo + lane * per + 32 * s + t;
     }
   }
+  const int base = n_stem + n_taken;
   for (int j = c_hi + lane; j < i; j += 32) out[base + (j - c_hi)] = j;
   const int total = base + (i - c_hi);
   for (int q = total + lane; q < a.k_max; q += 32) out[q] = -1;
@@ -172,10 +226,17 @@ cudaError_t launch_select_rows(const Plan& p, const float* M, int32_t* sel_idx, 
   a.stem = p.cfg.stem_blocks; a.local = p.cfg.local_blocks;
   const int64_t items = (int64_t)a.Hq * a.R_tot;
   const int grid = (int)((items + kThreads / 32 - 1) / (kThreads / 32));
+  constexpr int kSmem1 = (kThreads / 32) * 32 * 33 * 4, kSmem2 = (kThreads / 32) * 32 * 65 * 4;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
   if (p.max_nblk <= 1024)
-    select_rows_kernel<1><<<grid, kThreads, 0, s>>>(a);
+    select_rows_kernel<1><<<grid, kThreads, kSmem1, s>>>(a);
   else
-    select_rows_kernel<2><<<grid, kThreads, 0, s>>>(a);
+    select_rows_kernel<2><<<grid, kThreads, kSmem2, s>>>(a);
   return cudaGetLastError();
 }
 
