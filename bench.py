@@ -315,8 +315,8 @@ def main():
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
         "gpu_launches": main_res["launches_per_step"] * args.steps,
-        "stages_ms": {"pool": main_res["pool_ms"], "score_select": main_res["score_select_ms"],
-                      "pool_plus_score_select_one_call": main_res["scoring_stage_ms"],
+        "stages_ms": {"pool": main_res["pool_ms"], "metric_plus_select": main_res["score_select_ms"],
+                      "scoring_stage_one_call": main_res["scoring_stage_ms"],
                       "sparse_attention": main_res["attn_ms"], "dense_causal_same_kernel": main_res.get("dense_ms")},
         "effective_tflops": attn_tflops,
         "selected_over_causal_blocks": main_res["selected_blocks"] / main_res["causal_blocks"],
@@ -326,7 +326,7 @@ def main():
                                     f"nominal {NOMINAL['bf16_tflops']}",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal": attn_tflops / NOMINAL["bf16_tflops"]},
-        "roofline_scoring": {"kernels": "pool_kernel + score_select_kernel", "bound": "hbm", "achieved": score_gbs,
+        "roofline_scoring": {"kernels": "pool_kernel + metric_gemm_kernel + select_rows_kernel", "bound": "hbm", "achieved": score_gbs,
                              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": score_gbs / peaks["hbm_gbs"],
                              "frac_of_nominal": score_gbs / NOMINAL["hbm_gbs"], "bytes": main_res["score_bytes"],
                              "ms": score_ms},

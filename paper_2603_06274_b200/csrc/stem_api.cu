@@ -324,22 +324,24 @@ static int check_ws(const Plan& p, const void* ws, size_t bytes) {
 static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
 
 // Alg. 1 steps 1-3c on one stream: pooling (one pass over Q, K, V; also emits the pooled vectors as
-// bf16 parts), the metric of every causal block on the tensor cores into the workspace, and the
-// row-wise selection from it.
+// bf16 parts), the metric of every causal block on the tensor cores into the workspace (stored as
+// the selection's order-preserving keys), and the row-wise selection from it.
 // (Two ways of overlapping the HBM-bound pooling with the scoring were measured and dropped: phases
 // on two streams lose more to cross-stream event waits than they gain, and one persistent kernel
 // with a shared ticket list leaves too few warps per SM to stream HBM.)
 static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, uint8_t* w, int32_t* idx,
                                 int32_t* cnt, cudaStream_t s) {
   float* mv = (float*)(w + p.ws.mv);
-  float* M = (float*)(w + p.ws.metric);
-  int rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  float* M = (float*)(w + p.ws.metric);  // holds the selection keys of the metric, not the floats
+  int rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
+  if (rc != STEM_OK) return rc;
+  rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, (int32_t*)(w + p.ws.status), s));
+  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, true, true, (int32_t*)(w + p.ws.status), s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_select_rows(p, M, idx, cnt, s));
+  rc = cuda_rc(launch_select_rows(p, M, true, true, idx, cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }
@@ -355,11 +357,13 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   cudaStream_t s = (cudaStream_t)stream;
   p.last_launches = 0;
   float* mv = (float*)(w + p.ws.mv);
+  rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
+  if (rc != STEM_OK) return rc;
   rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   if (M) {
-    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, (int32_t*)(w + p.ws.status), s));
+    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, false, true, (int32_t*)(w + p.ws.status), s));
     if (rc != STEM_OK) return rc;
     p.last_launches++;
   }
@@ -377,15 +381,18 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
   p.last_launches = 0;
   cudaStream_t s = (cudaStream_t)stream;
   if (!M) {
-    // recompute the metric from the pooled vectors a previous stem_score left in the workspace
+    // recompute the metric (as selection keys) from the pooled vectors a previous stem_score left in the workspace
     float* Mw = (float*)(w + p.ws.metric);
-    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, (const float*)(w + p.ws.mv), Mw,
+    rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
+    if (rc != STEM_OK) return rc;
+    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, (const float*)(w + p.ws.mv), Mw, true, false,
                                     (int32_t*)(w + p.ws.status), s));
     if (rc != STEM_OK) return rc;
     p.last_launches++;
-    M = Mw;
+    rc = cuda_rc(launch_select_rows(p, Mw, true, true, sel_idx, sel_cnt, s));
+  } else {
+    rc = cuda_rc(launch_select_rows(p, M, false, false, sel_idx, sel_cnt, s));
   }
-  rc = cuda_rc(launch_select_rows(p, M, sel_idx, sel_cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }

@@ -81,8 +81,11 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
                         float* mv, void* qsplit, void* ksplit, cudaStream_t s);
 
 // Metric of every causal block (layout of stem_score's M) from the split pooled vectors, on the tensor cores.
+// as_keys: store the selection's order-preserving 32-bit keys of the values instead of the floats.
+// dependent: launch as a programmatic dependent of the kernel enqueued just before (its prologue overlaps that
+// kernel's tail).  The caller clears status words 4..7 beforehand.
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
-                               int32_t* status, cudaStream_t s);
+                               bool as_keys, bool dependent, int32_t* status, cudaStream_t s);
 
 // Shared-memory needs of the score/select kernel, for sizing its tiles at plan creation.
 size_t score_select_list_bytes(int k_max);   // per pooled query vector
@@ -97,7 +100,9 @@ cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, cons
 
 // Selection from a stored metric (layout of stem_score's M), one warp per (head, row).
 int row_select_max_blocks();  // largest supported N_blk of a sequence
-cudaError_t launch_select_rows(const Plan& p, const float* M, int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
+// is_keys: M holds the keys launch_metric_gemm(as_keys) wrote.
+cudaError_t launch_select_rows(const Plan& p, const float* M, bool is_keys, bool dependent, int32_t* sel_idx,
+                               int32_t* sel_cnt, cudaStream_t s);
 
 cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
                                     const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,

@@ -128,6 +128,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 
+// Monotone map float -> uint32 with -0 == +0 and NaN below everything (as -inf); every key is >= 1.
+__device__ __forceinline__ uint32_t metric_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  if ((u & 0x7fffffffu) > 0x7f800000u) u = 0xff800000u;  // NaN -> -inf
+  if (u == 0x80000000u) u = 0u;                          // -0 -> +0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 struct GemmArgs {
   const int32_t* tiles;  // [n_tiles][3] (sequence, row tile, column tile), column tile <= row tile
   const float* mv;       // [H_kv, R_tot]
@@ -137,6 +145,7 @@ struct GemmArgs {
   int64_t m_tot;
   int Hq, Hkv, g, R_tot;
   float beta, scale;
+  int as_keys;  // write order-preserving 32-bit keys of the metric (for the row selection) instead of floats
 };
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -166,6 +175,10 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Launched as a programmatic dependent of the pooling kernel, everything above overlaps its tail;
+  // its outputs are read only below this point.  (Without that launch attribute both are no-ops.)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   {
     const int c = threadIdx.x;  // bias of column c of the tile
     bias[c] = (tj * kTile + c < nb) ? a.beta * a.mv[(int64_t)kvh * a.R_tot + C0 + c] : 0.f;
@@ -236,6 +249,12 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         o.y = fmaf(a.scale, v[c4 * 4 + 1], bias[c + 1]);
         o.z = fmaf(a.scale, v[c4 * 4 + 2], bias[c + 2]);
         o.w = fmaf(a.scale, v[c4 * 4 + 3], bias[c + 3]);
+        if (a.as_keys) {
+          o.x = __uint_as_float(metric_key(o.x));
+          o.y = __uint_as_float(metric_key(o.y));
+          o.z = __uint_as_float(metric_key(o.z));
+          o.w = __uint_as_float(metric_key(o.w));
+        }
         *(float4*)(stage + m * kTile + (((c >> 2) ^ (m & 31)) << 2)) = o;
       }
     }
@@ -296,25 +315,33 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t planes) 
 }  // namespace
 
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
-                               int32_t* status, cudaStream_t s) {
+                               bool as_keys, bool dependent, int32_t* status, cudaStream_t s) {
   CUtensorMap mq, mk;
   if (!make_map(&mq, qsplit, p.R_tot, 3 * (int64_t)p.cfg.num_q_heads) ||
       !make_map(&mk, ksplit, p.R_tot, 3 * (int64_t)p.cfg.num_kv_heads))
     return cudaErrorInvalidValue;
   GemmArgs a{};
+  (void)status;
   a.tiles = p.d_gemm_tiles; a.mv = mv; a.M = M; a.status = status; a.rows = p.rows; a.m_tot = p.m_tot;
   a.Hq = p.cfg.num_q_heads; a.Hkv = p.cfg.num_kv_heads; a.g = a.Hq / a.Hkv; a.R_tot = p.R_tot;
-  a.beta = p.cfg.beta; a.scale = p.score_scale;
-  cudaError_t e0 = cudaMemsetAsync(status + 4, 0, 4 * sizeof(int32_t), s);  // this kernel's status words
-  if (e0 != cudaSuccess) return e0;
+  a.beta = p.cfg.beta; a.scale = p.score_scale; a.as_keys = as_keys ? 1 : 0;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(metric_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  metric_gemm_kernel<<<dim3((unsigned)p.n_gemm_tiles, (unsigned)a.Hq), kThreads, kSmemBytes, s>>>(mq, mk, a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)p.n_gemm_tiles, (unsigned)a.Hq);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, metric_gemm_kernel, mq, mk, a);
 }
 
 }  // namespace stem

@@ -41,6 +41,8 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
                                                    __nv_bfloat16* __restrict__ ksplit) {
   constexpr int kTokPerWarp = kBlock / 4;
   constexpr int kSteps = kTokPerWarp / 2;
+  // lets a kernel launched as a programmatic dependent set itself up during this kernel's last wave
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int slots = Hq + 2 * Hkv;
   const int R = blockIdx.x / slots;
   const int slot = blockIdx.x - R * slots;

@@ -82,7 +82,7 @@ __device__ __forceinline__ uint32_t lowest_bits(uint32_t m, int n) {
 }
 
 // SETS = 32-key register sets per lane: rows of up to SETS * 1024 candidates.
-template <int SETS>
+template <int SETS, bool KEYS>
 __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kernel(const SelArgs a) {
   constexpr int kStride = 32 * SETS + 1;  // words of shared memory per lane (odd: conflict-free both ways)
   extern __shared__ uint32_t stage_all[];
@@ -110,12 +110,14 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
 #pragma unroll
   for (int s = 0; s < SETS; ++s) sel[s] = 0u;
 
+  // Launched as a programmatic dependent of the metric kernel, the set-up above overlaps its tail.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (need > 0) {
     // ---- keys: coalesced loads, through shared memory into runs of `per` consecutive candidates per lane
     const uint32_t magic = ((1u << 20) + per - 1) / per;  // q / per == (q * magic) >> 20 for q < 2048
     for (int q = lane; q < n_cand; q += 32) {
       const uint32_t owner = ((uint32_t)q * magic) >> 20;
-      stage[owner * kStride + (q - owner * per)] = metric_key(mrow[q]);
+      stage[owner * kStride + (q - owner * per)] = KEYS ? __float_as_uint(mrow[q]) : metric_key(mrow[q]);
     }
     __syncwarp();
     uint32_t tw[SETS][32];
@@ -219,7 +221,8 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
 
 int row_select_max_blocks() { return 2 * 1024; }
 
-cudaError_t launch_select_rows(const Plan& p, const float* M, int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
+cudaError_t launch_select_rows(const Plan& p, const float* M, bool is_keys, bool dependent, int32_t* sel_idx,
+                               int32_t* sel_cnt, cudaStream_t s) {
   SelArgs a{};
   a.M = M; a.sel_idx = sel_idx; a.sel_cnt = sel_cnt; a.rows = p.rows; a.m_tot = p.m_tot;
   a.Hq = p.cfg.num_q_heads; a.R_tot = p.R_tot; a.k_max = p.k_max;
@@ -229,15 +232,27 @@ cudaError_t launch_select_rows(const Plan& p, const float* M, int32_t* sel_idx, 
   constexpr int kSmem1 = (kThreads / 32) * 32 * 33 * 4, kSmem2 = (kThreads / 32) * 32 * 65 * 4;
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
+    cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(select_rows_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  if (p.max_nblk <= 1024)
-    select_rows_kernel<1><<<grid, kThreads, kSmem1, s>>>(a);
-  else
-    select_rows_kernel<2><<<grid, kThreads, kSmem2, s>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent ? 1 : 0;
+  if (p.max_nblk <= 1024) {
+    cfg.dynamicSmemBytes = kSmem1;
+    return is_keys ? cudaLaunchKernelEx(&cfg, select_rows_kernel<1, true>, a) : cudaLaunchKernelEx(&cfg, select_rows_kernel<1, false>, a);
+  }
+  cfg.dynamicSmemBytes = kSmem2;
+  return is_keys ? cudaLaunchKernelEx(&cfg, select_rows_kernel<2, true>, a) : cudaLaunchKernelEx(&cfg, select_rows_kernel<2, false>, a);
 }
 
 }  // namespace stem
