@@ -626,8 +626,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       while (ok && (has0 || has1)) {
         const bool p0 = try_load(c0, has0, ord0, 0);
         const bool p1 = try_load(c1, has1, ord1, 1);
-        if (p0 || p1) { t0 = globaltimer(); spin = 0; }
-        else if ((++spin & 31u) == 0u) {
+        if (p0 || p1) { t0 = globaltimer(); spin = 0; continue; }
+        __nanosleep(400);  // a Q tile is wanted once per item: poll slowly, the issue slots belong to the softmax warps
+        if ((++spin & 31u) == 0u) {
           bool stop = *abort_flag != 0;
           if (!stop && globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); stop = true; }
           if (__any_sync(0xffffffffu, stop)) ok = false;
