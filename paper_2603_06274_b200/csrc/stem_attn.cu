@@ -877,13 +877,15 @@ cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K,
 
   cudaError_t e = cudaMemsetAsync(status, 0, kStatusWords * sizeof(int32_t), s);
   if (e != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the attribute belongs to the device's context: set it once per device of this process
+  static bool attr_set[64] = {};
+  const int dev_slot = p.device & 63;
+  if (!attr_set[dev_slot]) {
     e = cudaFuncSetAttribute(sparse_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(sparse_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev_slot] = true;
   }
   const int grid = std::min(p.n_items, p.sm_count);
   if (B == 128)

@@ -325,11 +325,13 @@ cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ks
   a.tiles = p.d_gemm_tiles; a.mv = mv; a.M = M; a.status = status; a.rows = p.rows; a.m_tot = p.m_tot;
   a.Hq = p.cfg.num_q_heads; a.Hkv = p.cfg.num_kv_heads; a.g = a.Hq / a.Hkv; a.R_tot = p.R_tot;
   a.beta = p.cfg.beta; a.scale = p.score_scale; a.as_keys = as_keys ? 1 : 0;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the attribute belongs to the device's context: set it once per device of this process
+  static bool attr_set[64] = {};
+  const int dev_slot = p.device & 63;
+  if (!attr_set[dev_slot]) {
     cudaError_t e = cudaFuncSetAttribute(metric_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev_slot] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)p.n_gemm_tiles, (unsigned)a.Hq);

@@ -230,13 +230,15 @@ cudaError_t launch_select_rows(const Plan& p, const float* M, bool is_keys, bool
   const int64_t items = (int64_t)a.Hq * a.R_tot;
   const int grid = (int)((items + kThreads / 32 - 1) / (kThreads / 32));
   constexpr int kSmem1 = (kThreads / 32) * 32 * 33 * 4, kSmem2 = (kThreads / 32) * 32 * 65 * 4;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the attribute belongs to the device's context: set it once per device of this process
+  static bool attr_set[64] = {};
+  const int dev_slot = p.device & 63;
+  if (!attr_set[dev_slot]) {
     cudaError_t e = cudaFuncSetAttribute(select_rows_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(select_rows_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev_slot] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);

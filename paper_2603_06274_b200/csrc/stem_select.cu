@@ -454,11 +454,13 @@ cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, cons
   a.nq_slots = (p.sel_nq + 7) / 8 * 8;
   const size_t smem = score_select_fixed_smem() + (size_t)a.nq_slots * score_select_list_bytes(p.k_max);
   if (smem > 227 * 1024 || p.max_nblk > kMaxWords * 32) return cudaErrorInvalidValue;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the attribute belongs to the device's context: set it once per device of this process
+  static bool attr_set[64] = {};
+  const int dev_slot = p.device & 63;
+  if (!attr_set[dev_slot]) {
     cudaError_t e = cudaFuncSetAttribute(score_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev_slot] = true;
   }
   const dim3 grid((unsigned)p.n_sel_tiles * (unsigned)a.Hkv);
   score_select_kernel<<<grid, kThreads, smem, s>>>(a);
