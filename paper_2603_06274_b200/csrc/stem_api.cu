@@ -113,9 +113,9 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
 
   std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_len(batch), seq_nblk(batch),
       seq_row_off(batch);
-  std::vector<int64_t> seq_m_off(batch);
+  std::vector<int64_t> seq_m_off(batch), seq_mt_off(batch);
   std::vector<int32_t> seq_kt_off(batch);
-  int64_t m_off = 0;
+  int64_t m_off = 0, mt_off = 0;
   for (int b = 0; b < batch; ++b) {
     const int32_t n = p.cu[b + 1] - p.cu[b];
     const int32_t nb = (n + B - 1) / B;
@@ -124,6 +124,8 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     seq_nblk[b] = nb;
     seq_row_off[b] = (int32_t)row_seq.size();
     seq_m_off[b] = m_off;
+    seq_mt_off[b] = mt_off;
+    mt_off += (int64_t)nb * ((nb + 31) / 32 * 32);  // rows padded to whole 32-column groups
     seq_kt_off[b] = p.kt_width;
     p.kt_width += (nb + 63) / 64 * 64;
     m_off += (int64_t)nb * nb;
@@ -147,6 +149,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   }
   p.R_tot = (int32_t)row_seq.size();
   p.m_tot = m_off;
+  p.mt_tot = mt_off;
   p.selected_blocks *= Hq;
   p.causal_blocks *= Hq;
   p.selected_pairs *= Hq;
@@ -218,7 +221,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
     p.ws.qsplit = off; off = align_up(off + (size_t)3 * Hq * p.R_tot * kHeadDim * 2, 256);
     p.ws.ksplit = off; off = align_up(off + (size_t)3 * Hkv * p.R_tot * kHeadDim * 2, 256);
-    p.ws.metric = off; off = align_up(off + (size_t)Hq * (size_t)p.m_tot * 4, 256);
+    p.ws.metric = off; off = align_up(off + (size_t)Hq * (size_t)p.mt_tot * 4, 256);
     p.ws.sel_idx = off; off = align_up(off + (size_t)Hq * p.R_tot * p.k_max * 4, 256);
     p.ws.sel_cnt = off; off = align_up(off + (size_t)Hq * p.R_tot * 4, 256);
     p.ws.total = off;
@@ -235,7 +238,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   const size_t o_row_seq = push(blob, row_seq), o_row_r = push(blob, row_r), o_row_tok0 = push(blob, row_tok0),
                o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
                o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
-               o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off),
+               o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off), o_seq_mt_off = push(blob, seq_mt_off),
                o_seq_kt_off = push(blob, seq_kt_off),
                o_tiles = push(blob, tiles), o_gt = push(blob, gemm_tiles), o_ws = push(blob, work_sparse),
                o_wd = push(blob, work_dense);
@@ -257,6 +260,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.rows.seq_nblk = (const int32_t*)(d + o_seq_nblk);
   p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
+  p.rows.seq_mt_off = (const int64_t*)(d + o_seq_mt_off);
   p.rows.seq_kt_off = (const int32_t*)(d + o_seq_kt_off);
   p.d_sel_tiles = (const int32_t*)(d + o_tiles);
   p.d_gemm_tiles = (const int32_t*)(d + o_gt);
@@ -325,14 +329,14 @@ static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR
 
 // Alg. 1 steps 1-3c on one stream: pooling (one pass over Q, K, V; also emits the pooled vectors as
 // bf16 parts), the metric of every causal block on the tensor cores into the workspace (stored as
-// the selection's order-preserving keys), and the row-wise selection from it.
+// bit planes of the selection's order-preserving keys), and the row-wise selection from it.
 // (Two ways of overlapping the HBM-bound pooling with the scoring were measured and dropped: phases
 // on two streams lose more to cross-stream event waits than they gain, and one persistent kernel
 // with a shared ticket list leaves too few warps per SM to stream HBM.)
 static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, uint8_t* w, int32_t* idx,
                                 int32_t* cnt, cudaStream_t s) {
   float* mv = (float*)(w + p.ws.mv);
-  float* M = (float*)(w + p.ws.metric);  // holds the selection keys of the metric, not the floats
+  float* M = (float*)(w + p.ws.metric);  // holds the bit planes of the selection keys, not the floats
   int rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
   rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
@@ -341,7 +345,7 @@ static int enqueue_score_select(const Plan& p, const void* Q, const void* K, con
   rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, true, true, (int32_t*)(w + p.ws.status), s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_select_rows(p, M, true, true, idx, cnt, s));
+  rc = cuda_rc(launch_select_planes(p, (const uint32_t*)M, true, idx, cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }
@@ -389,9 +393,9 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
                                     (int32_t*)(w + p.ws.status), s));
     if (rc != STEM_OK) return rc;
     p.last_launches++;
-    rc = cuda_rc(launch_select_rows(p, Mw, true, true, sel_idx, sel_cnt, s));
+    rc = cuda_rc(launch_select_planes(p, (const uint32_t*)Mw, true, sel_idx, sel_cnt, s));
   } else {
-    rc = cuda_rc(launch_select_rows(p, M, false, false, sel_idx, sel_cnt, s));
+    rc = cuda_rc(launch_select_rows(p, M, false, sel_idx, sel_cnt, s));
   }
   if (rc == STEM_OK) p.last_launches++;
   return rc;

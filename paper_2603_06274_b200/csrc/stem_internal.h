@@ -29,6 +29,7 @@ struct RowTables {
   const int32_t* seq_nblk;     // [batch]
   const int32_t* seq_row_off;  // [batch] global row of the sequence's row 0
   const int64_t* seq_m_off;    // [batch] offset of the sequence's square inside one head of M
+  const int64_t* seq_mt_off;   // [batch] offset of the sequence inside one head of the bit-plane metric
   const int32_t* seq_kt_off;   // [batch] first column of the sequence inside a row of Kbar^T (multiple of 64)
 };
 
@@ -38,7 +39,7 @@ struct WorkspaceLayout {
   size_t mv = 0;       // fp32 [H_kv, R_tot]
   size_t qsplit = 0;   // bf16 [3, H_q, R_tot, d]: Qbar as hi + mid + lo parts
   size_t ksplit = 0;   // bf16 [3, H_kv, R_tot, d]: Kbar likewise (row = global block row)
-  size_t metric = 0;   // fp32 [H_q, m_tot]: M of the fused path
+  size_t metric = 0;   // uint32 [H_q, mt_tot]: the metric of the fused path as bit planes of its selection keys
   size_t sel_idx = 0;  // int32 [H_q, R_tot, k_max]
   size_t sel_cnt = 0;  // int32 [H_q, R_tot]
   size_t total = 0;
@@ -52,6 +53,7 @@ struct Plan {
   int32_t T = 0, R_tot = 0, k_max = 0, max_nblk = 0;
   int32_t kt_width = 0;  // row length of Kbar^T: sum over sequences of N_blk rounded up to 64
   int64_t m_tot = 0;
+  int64_t mt_tot = 0;  // words per head of the bit-plane metric: sum_b N_blk(b) * roundup(N_blk(b), 32)
   int64_t selected_blocks = 0, causal_blocks = 0, selected_pairs = 0, causal_pairs = 0;
   std::vector<int32_t> k_eff;  // host copy [R_tot]
   float score_scale = 1.f, softmax_scale = 0.f;
@@ -81,7 +83,9 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
                         float* mv, void* qsplit, void* ksplit, cudaStream_t s);
 
 // Metric of every causal block (layout of stem_score's M) from the split pooled vectors, on the tensor cores.
-// as_keys: store the selection's order-preserving 32-bit keys of the values instead of the floats.
+// as_keys: instead of the floats, store bit planes of the selection's order-preserving keys: row r of sequence b at
+// seq_mt_off[b] + r * roundup(N_blk(b), 32), and in it, for every group of 32 columns, 32 words, word k holding bit k
+// of the 32 keys (bit t <-> column 32 * group + t).  What launch_select_planes reads.
 // dependent: launch as a programmatic dependent of the kernel enqueued just before (its prologue overlaps that
 // kernel's tail).  The caller clears status words 4..7 beforehand.
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
@@ -100,9 +104,11 @@ cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, cons
 
 // Selection from a stored metric (layout of stem_score's M), one warp per (head, row).
 int row_select_max_blocks();  // largest supported N_blk of a sequence
-// is_keys: M holds the keys launch_metric_gemm(as_keys) wrote.
-cudaError_t launch_select_rows(const Plan& p, const float* M, bool is_keys, bool dependent, int32_t* sel_idx,
-                               int32_t* sel_cnt, cudaStream_t s);
+cudaError_t launch_select_rows(const Plan& p, const float* M, bool dependent, int32_t* sel_idx, int32_t* sel_cnt,
+                               cudaStream_t s);
+// The same selection from the bit-plane metric launch_metric_gemm(as_keys) wrote.
+cudaError_t launch_select_planes(const Plan& p, const uint32_t* Mt, bool dependent, int32_t* sel_idx, int32_t* sel_cnt,
+                                 cudaStream_t s);
 
 cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
                                     const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,

@@ -136,16 +136,45 @@ __device__ __forceinline__ uint32_t metric_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// In-register transpose of a 32 x 32 bit matrix: afterwards bit t of w[b] is bit b of the old w[t].
+__device__ __forceinline__ void transpose32(uint32_t (&w)[32]) {
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {  // 16-bit halves: byte permutes
+    const uint32_t lo = __byte_perm(w[k], w[k + 16], 0x5410), hi = __byte_perm(w[k], w[k + 16], 0x7632);
+    w[k] = lo;
+    w[k + 16] = hi;
+  }
+#pragma unroll
+  for (int k = 0; k < 32; ++k) {  // bytes
+    if (k & 8) continue;
+    const uint32_t lo = __byte_perm(w[k], w[k + 8], 0x6240), hi = __byte_perm(w[k], w[k + 8], 0x7351);
+    w[k] = lo;
+    w[k + 8] = hi;
+  }
+#pragma unroll
+  for (int s = 2; s < 5; ++s) {
+    const int j = 16 >> s;
+    const uint32_t mhi = s == 2 ? 0xf0f0f0f0u : s == 3 ? 0xccccccccu : 0xaaaaaaaau;
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      if (k & j) continue;
+      const uint32_t x = w[k], y = w[k + j];
+      w[k] = (x & ~mhi) | ((y << j) & mhi);
+      w[k + j] = ((x >> j) & ~mhi) | (y & mhi);
+    }
+  }
+}
+
 struct GemmArgs {
   const int32_t* tiles;  // [n_tiles][3] (sequence, row tile, column tile), column tile <= row tile
   const float* mv;       // [H_kv, R_tot]
   float* M;
   int32_t* status;
   RowTables rows;
-  int64_t m_tot;
+  int64_t m_tot, mt_tot;
   int Hq, Hkv, g, R_tot;
   float beta, scale;
-  int as_keys;  // write order-preserving 32-bit keys of the metric (for the row selection) instead of floats
+  int as_keys;  // write bit planes of the metric's selection keys (for launch_select_planes) instead of floats
 };
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -232,7 +261,31 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   ok = mbar_wait(bar_done, 0, a.status) && ok;
   ok = __syncthreads_and(ok);
   float* stage = (float*)smem_gen;  // 128 x 128 fp32 over the operand tiles, which are no longer needed
-  if (ok) {
+  if (ok && a.as_keys) {
+    // For the selection: each thread turns the keys of its row, 32 columns at a time, into 32 bit
+    // planes (word k = bit k of the 32 keys) and stores them as one 128-byte line of the row.
+    tc_fence_after();
+    const int m = warp * 32 + lane;
+    const int r = ti * kTile + m;
+    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+    const int stride = (nb + 31) & ~31;
+    uint32_t* dst = (uint32_t*)a.M + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)r * stride + tj * kTile;
+#pragma unroll 1
+    for (int gq = 0; gq < 4; ++gq) {
+      float v[32];
+      tmem_ld32(taddr + gq * 32, v);
+      tmem_ld_wait();
+      uint32_t w[32];
+#pragma unroll
+      for (int c = 0; c < 32; ++c) w[c] = metric_key(fmaf(a.scale, v[c], bias[gq * 32 + c]));
+      transpose32(w);
+      if (r < nb && tj * kTile + gq * 32 < stride) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *(uint4*)(dst + gq * 32 + q * 4) = make_uint4(w[q * 4], w[q * 4 + 1], w[q * 4 + 2], w[q * 4 + 3]);
+      }
+    }
+  } else if (ok) {
     tc_fence_after();
     const int m = warp * 32 + lane;  // row of the tile == TMEM lane
     const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
@@ -249,12 +302,6 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         o.y = fmaf(a.scale, v[c4 * 4 + 1], bias[c + 1]);
         o.z = fmaf(a.scale, v[c4 * 4 + 2], bias[c + 2]);
         o.w = fmaf(a.scale, v[c4 * 4 + 3], bias[c + 3]);
-        if (a.as_keys) {
-          o.x = __uint_as_float(metric_key(o.x));
-          o.y = __uint_as_float(metric_key(o.y));
-          o.z = __uint_as_float(metric_key(o.z));
-          o.w = __uint_as_float(metric_key(o.w));
-        }
         *(float4*)(stage + m * kTile + (((c >> 2) ^ (m & 31)) << 2)) = o;
       }
     }
@@ -265,7 +312,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(128) : "memory");
   }
-  if (!ok) return;
+  if (!ok || a.as_keys) return;
   // ---- causal part of the tile to M, one row per step of a warp, 128 contiguous bytes per store
   float* mseq = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq];
   for (int mm = 0; mm < 32; ++mm) {
@@ -322,7 +369,7 @@ cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ks
     return cudaErrorInvalidValue;
   GemmArgs a{};
   (void)status;
-  a.tiles = p.d_gemm_tiles; a.mv = mv; a.M = M; a.status = status; a.rows = p.rows; a.m_tot = p.m_tot;
+  a.tiles = p.d_gemm_tiles; a.mv = mv; a.M = M; a.status = status; a.rows = p.rows; a.m_tot = p.m_tot; a.mt_tot = p.mt_tot;
   a.Hq = p.cfg.num_q_heads; a.Hkv = p.cfg.num_kv_heads; a.g = a.Hq / a.Hkv; a.R_tot = p.R_tot;
   a.beta = p.cfg.beta; a.scale = p.score_scale; a.as_keys = as_keys ? 1 : 0;
   // the attribute belongs to the device's context: set it once per device of this process
