@@ -275,10 +275,17 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       float v[32];
       tmem_ld32(taddr + gq * 32, v);
       tmem_ld_wait();
+      // key = bits ^ (negative ? all ones : sign bit) of the value with -0 -> +0 and NaN -> -inf; the
+      // exclusive-or is applied to the planes (32 operations for 32 keys) instead of to the keys
       uint32_t w[32];
 #pragma unroll
-      for (int c = 0; c < 32; ++c) w[c] = metric_key(fmaf(a.scale, v[c], bias[gq * 32 + c]));
+      for (int c = 0; c < 32; ++c)
+        w[c] = __float_as_uint(fmaxf(fmaf(a.scale, v[c], bias[gq * 32 + c]) + 0.0f, __int_as_float(0xff800000)));
       transpose32(w);
+      const uint32_t neg = w[31];  // bit t: value t is negative
+#pragma unroll
+      for (int k = 0; k < 31; ++k) w[k] ^= neg;
+      w[31] = ~neg;
       if (r < nb && tj * kTile + gq * 32 < stride) {
 #pragma unroll
         for (int q = 0; q < 8; ++q)

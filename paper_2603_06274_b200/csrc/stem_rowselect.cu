@@ -9,8 +9,7 @@
 // every lane holds a run of consecutive candidates (lane L the candidates L*c .. L*c + c - 1,
 // c = ceil(n_cand / 32)).  Each lane bit-transposes its keys (word b = bit b of every key of the
 // lane), and the need-th largest key is found by a most-significant-bit-first radix descent that
-// costs one AND + popc per lane and one warp reduction per varying key bit, and stops as soon as
-// the keys still undecided are exactly the ones still needed.  The selected ids come out in
+// costs one AND + popc per lane and one warp reduction per key bit.  The selected ids come out in
 // ascending order by a warp prefix sum over the lanes' counts.  The kernel is bound by the integer
 // pipe, so the stages are written for few logic instructions (byte permutes in the transpose).
 #include <cuda_runtime.h>
@@ -121,8 +120,6 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
     __syncwarp();
     uint32_t tw[SETS][32];
     uint32_t act[SETS], gt[SETS];  // still in the descent / known to be above the threshold
-    uint32_t vary = 0u;
-    const uint32_t key0 = stage[0];
     const int mine = min(max(n_cand - lane * per, 0), per);  // candidates of this lane
 #pragma unroll
     for (int s = 0; s < SETS; ++s) {
@@ -135,7 +132,6 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
         if (32 * s + t < per) {  // warp-uniform
           kx = stage[lane * kStride + 32 * s + t];
           if (32 * s + t >= mine) kx = 0u;
-          else vary |= kx ^ key0;
         }
         tw[s][t] = kx;
       }
@@ -143,27 +139,24 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
     }
 
     // ---- the need-th largest key by radix descent; gt = keys above it, act = keys still undecided.
-    // The descent stops deciding as soon as the undecided keys are exactly the ones still needed
-    // (at once when every candidate is needed); at the end the undecided keys are all equal.
-    vary = __reduce_or_sync(0xffffffffu, vary);
-    int k = need, na = n_cand;  // rank wanted among the undecided keys, number of undecided keys
+    // Straight-line over all 32 bits (a bit all undecided keys agree on changes nothing: its count is
+    // 0 or all of them); at the end the undecided keys are all equal.  The loop is kept free of
+    // branches: with warp-uniform branches around the warp reduction in the unrolled loop this
+    // compiler produced wrong lists.
+    int k = need;  // rank wanted among the undecided keys
 #pragma unroll
     for (int b = 31; b >= 0; --b) {
-      if (((vary >> b) & 1u) != 0u && k != na) {  // warp-uniform; a bit all candidates agree on decides nothing
-        int cnt = 0;
+      int cnt = 0;
 #pragma unroll
-        for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
-        cnt = __reduce_add_sync(0xffffffffu, cnt);
-        if (cnt >= k) {
-          na = cnt;
+      for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      const bool inside = cnt >= k;  // the k-th largest has this bit set
+      k -= inside ? 0 : cnt;
 #pragma unroll
-          for (int s = 0; s < SETS; ++s) act[s] &= tw[s][b];
-        } else {
-          k -= cnt;
-          na -= cnt;
-#pragma unroll
-          for (int s = 0; s < SETS; ++s) { gt[s] |= act[s] & tw[s][b]; act[s] &= ~tw[s][b]; }
-        }
+      for (int s = 0; s < SETS; ++s) {
+        const uint32_t ones = act[s] & tw[s][b];
+        gt[s] |= inside ? 0u : ones;
+        act[s] = inside ? ones : (act[s] ^ ones);
       }
     }
     const int rem = k;  // of the undecided keys the first `rem` by block id are taken
@@ -258,7 +251,6 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_planes_ker
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (need > 0) {
     uint32_t tw[SETS][32], act[SETS], gt[SETS];
-    uint32_t has1 = 0u, has0 = 0u;  // bit k: some candidate of this lane has key bit k set / clear
 #pragma unroll
     for (int s = 0; s < SETS; ++s) {
       const int j0 = 32 * (lane + 32 * s);  // first column of this lane's group
@@ -277,32 +269,25 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_planes_ker
 #pragma unroll
         for (int k = 0; k < 32; ++k) tw[s][k] = 0u;
       }
-#pragma unroll
-      for (int k = 0; k < 32; ++k) {
-        if (tw[s][k] & act[s]) has1 |= 1u << k;
-        if (~tw[s][k] & act[s]) has0 |= 1u << k;
-      }
     }
-    const uint32_t vary = __reduce_or_sync(0xffffffffu, has1) & __reduce_or_sync(0xffffffffu, has0);
-    // radix descent as in select_rows_kernel
-    int k = need, na = n_cand;
+    // Radix descent as in select_rows_kernel, over all 32 bits: a bit all undecided keys agree on
+    // changes nothing (its count is 0 or all of them), so the bits need not be screened first.
+    int k = need;
 #pragma unroll
     for (int b = 31; b >= 0; --b) {
-      if (((vary >> b) & 1u) != 0u && k != na) {
-        int cnt = 0;
+      // straight-line step: keys with the bit set are either where the k-th largest lies (cnt >= k)
+      // or all above it
+      int cnt = 0;
 #pragma unroll
-        for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
-        cnt = __reduce_add_sync(0xffffffffu, cnt);
-        if (cnt >= k) {
-          na = cnt;
+      for (int s = 0; s < SETS; ++s) cnt += __popc(tw[s][b] & act[s]);
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      const bool inside = cnt >= k;
+      k -= inside ? 0 : cnt;
 #pragma unroll
-          for (int s = 0; s < SETS; ++s) act[s] &= tw[s][b];
-        } else {
-          k -= cnt;
-          na -= cnt;
-#pragma unroll
-          for (int s = 0; s < SETS; ++s) { gt[s] |= act[s] & tw[s][b]; act[s] &= ~tw[s][b]; }
-        }
+      for (int s = 0; s < SETS; ++s) {
+        const uint32_t ones = act[s] & tw[s][b];
+        gt[s] |= inside ? 0u : ones;
+        act[s] = inside ? ones : (act[s] ^ ones);
       }
     }
     // of the undecided keys the first k in column order (set-major, then lane, then bit) are taken
