@@ -76,3 +76,19 @@ def test_long_candidate_lists():
     w = wl.small("long_lists", seqlens=(400 * 128,), hq=2, hkv=1, block=128, permille=500)
     data, q, k, v = _dev(w)
     check_full_path(w, data, q, k, v, n_random=6)
+
+
+def test_equal_metrics_are_broken_by_block_id_in_the_fused_path():
+    # every K token and every V token of a kv head is the same vector: a row's candidates all have the same
+    # metric (also on the GPU: each column of the contraction sees the same operands), so the budget must go to the
+    # candidates with the smallest block ids, in the fused path's bit-plane selection kernel too
+    w = wl.small("all_ties", seqlens=(6000,), hq=4, hkv=2, block=64, permille=300)
+    data = wl.make_qkv(w)
+    data["k"][:] = data["k"][0:1]
+    data["v"][:] = data["v"][0:1]
+    q, k, v = to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"])
+    idx_g, cnt_g, _ = check_full_path(w, data, q, k, v, tie_budget=0)
+    r = 80                                                     # 81 causal blocks, 4 + 4 forced
+    n = int(cnt_g[1, r])
+    want = np.concatenate([np.arange(0, n - w.local_blocks), np.arange(r + 1 - w.local_blocks, r + 1)])
+    assert np.array_equal(idx_g[1, r, :n], want)
