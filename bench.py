@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # DRAM traffic of one sparse-attention launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum),
 # captured on the workload itself; a workload without a capture reports null.
-NCU_ATTN_DRAM_BYTES_PER_LAUNCH = {"cfg3_llama3_8b_128k": 1664264704 + 1042041856}
+NCU_ATTN_DRAM_BYTES_PER_LAUNCH = {"cfg3_llama3_8b_128k": 1660022528 + 1041437440}
 
 
 def load_peaks():
@@ -326,7 +326,7 @@ def main():
                                     f"nominal {NOMINAL['bf16_tflops']}",
                      "frac_of_sustained": attn_tflops / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal": attn_tflops / NOMINAL["bf16_tflops"]},
-        "roofline_scoring": {"kernels": "pool_kernel + metric_gemm_kernel + select_rows_kernel", "bound": "hbm", "achieved": score_gbs,
+        "roofline_scoring": {"kernels": "pool_kernel + metric_gemm_kernel + select_planes_kernel", "bound": "hbm", "achieved": score_gbs,
                              "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": score_gbs / peaks["hbm_gbs"],
                              "frac_of_nominal": score_gbs / NOMINAL["hbm_gbs"], "bytes": main_res["score_bytes"],
                              "ms": score_ms},

@@ -14,8 +14,10 @@
 // One CTA per (128 x 128 tile of one sequence's causal triangle, query head), two CTAs per SM: TMA
 // brings the 3 + 3 operand parts (K-major, 128-byte swizzle) one half of the head dimension at a
 // time, one thread issues the 2 x 24 MMAs, the four warps
-// read the accumulator (one row per thread), apply scale and bias, turn the tile through shared
-// memory and write the causal part of it with coalesced stores.  Waits are bounded.
+// read the accumulator (one row per thread), apply scale and bias, and either turn the tile through
+// shared memory and write the causal part of it with coalesced stores (the public M), or write each
+// row's selection keys as bit planes, one 128-byte line per 32 columns (the fused path's workspace
+// form, read by the bit-plane selection kernel).  Waits are bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

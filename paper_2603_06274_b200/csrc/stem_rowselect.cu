@@ -5,13 +5,16 @@
 // causal blocks between them.  The row takes the need = k_eff(r) - #forced best candidates by
 // (metric descending, block id ascending), metric compared as an order-preserving 32-bit key with
 // -0 == +0 and NaN as -inf.
-// The warp reads the row's metric with coalesced loads and turns it through shared memory so that
-// every lane holds a run of consecutive candidates (lane L the candidates L*c .. L*c + c - 1,
-// c = ceil(n_cand / 32)).  Each lane bit-transposes its keys (word b = bit b of every key of the
-// lane), and the need-th largest key is found by a most-significant-bit-first radix descent that
-// costs one AND + popc per lane and one warp reduction per key bit.  The selected ids come out in
-// ascending order by a warp prefix sum over the lanes' counts.  The kernel is bound by the integer
-// pipe, so the stages are written for few logic instructions (byte permutes in the transpose).
+// Each lane holds a run of consecutive blocks of the row as bit planes (word b = bit b of every key
+// of the lane), and the need-th largest key is found by a most-significant-bit-first radix descent
+// that costs one AND + popc per lane and one warp reduction per key bit.  The selected ids come out
+// in ascending order by a warp prefix sum over the lanes' counts.  Two kernels:
+//   select_rows_kernel    from float metrics (the public M): coalesced loads, a turn through shared
+//                         memory into lane-contiguous runs of candidates, key conversion and an
+//                         in-register bit transpose per lane;
+//   select_planes_kernel  from the bit planes the metric kernel writes for the fused path: one
+//                         128-byte line per lane, nothing to convert or transpose.
+// Both are bound by the integer pipe, so the stages are written for few logic instructions.
 #include <cuda_runtime.h>
 
 #include "stem_internal.h"
