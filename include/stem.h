@@ -179,7 +179,8 @@ int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void
 /* Synchronises `stream`, then reads and clears the device status words of `workspace`.
  * Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in a kernel gave up; outputs of that
  * call are undefined) or STEM_ERR_CUDA.  detail (optional, HOST int32[4]) receives the raw words:
- * {code, block index, role, barrier id}. */
+ * {code, block index, role, barrier id} of the attention kernel (code 1), or {2, tile, head, 0} when
+ * the wait that gave up was in the metric kernel. */
 int stem_check_status(const stem_plan* plan, void* workspace, void* stream, int32_t* detail_host);
 
 /* Number of kernels the last hot call on this plan launched (for launch accounting). */

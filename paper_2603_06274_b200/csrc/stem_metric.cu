@@ -32,8 +32,8 @@ constexpr int kTile = 128;
 constexpr int kPartBytes = kTile * 128;               // one operand part, one 64-column half of d (bf16): 16 KB
 constexpr int kSmemOps = 6 * kPartBytes;              // A hi/mid/lo, B hi/mid/lo (reused for both halves of d)
 constexpr int kSmemBias = kSmemOps;                   // 128 floats
-constexpr int kSmemBars = kSmemBias + kTile * 4;      // full, half_done, done
-constexpr int kSmemTmem = kSmemBars + 32;
+constexpr int kSmemBars = kSmemBias + kTile * 4;      // full[3], half_done, done
+constexpr int kSmemTmem = kSmemBars + 48;
 constexpr int kSmemTotal = kSmemTmem + 16;
 constexpr int kSmemBytes = kSmemTotal + 1024;         // slack for manual 1024-byte alignment; two CTAs per SM
 static_assert(kTile * kTile * 4 <= kSmemOps, "the output tile is staged over the operand tiles");
@@ -185,7 +185,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - (uint32_t)__cvta_generic_to_shared(smem_raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t bar_full = smem_base + kSmemBars, bar_half = bar_full + 8, bar_done = bar_full + 16;
+  const uint32_t bar_full = smem_base + kSmemBars, bar_half = bar_full + 24, bar_done = bar_full + 32;  // bar_full: 3 barriers
   float* bias = (float*)(smem_gen + kSmemBias);
 
   const int seq = a.tiles[3 * blockIdx.x], ti = a.tiles[3 * blockIdx.x + 1], tj = a.tiles[3 * blockIdx.x + 2];
@@ -196,6 +196,8 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
   if (threadIdx.x == 0) {
     mbar_init(bar_full, 1);
+    mbar_init(bar_full + 8, 1);
+    mbar_init(bar_full + 16, 1);
     mbar_init(bar_half, 1);
     mbar_init(bar_done, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -231,21 +233,26 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     for (int half = 0; half < 2 && ok; ++half) {
       if (half == 1) ok = __all_sync(0xffffffffu, mbar_wait(bar_half, 0, a.status));  // the first half's MMAs have read the parts
       if (!ok) break;
+      // The copies go out in the order the products need them, two parts per barrier, so that the
+      // MMAs start when the first third of the bytes has landed.
+      constexpr int kLoadA[3] = {1, 0, 2}, kLoadB[3] = {1, 2, 0};
       if (leader) {
-        mbar_expect_tx(bar_full, kSmemOps);
 #pragma unroll
-        for (int s = 0; s < 3; ++s) {
-          tma_load_3d(smem_base + s * kPartBytes, &map_q, bar_full, 64 * half, R0, s * a.Hq + h);
-          tma_load_3d(smem_base + (3 + s) * kPartBytes, &map_k, bar_full, 64 * half, C0, s * a.Hkv + kvh);
+        for (int q = 0; q < 3; ++q) {
+          mbar_expect_tx(bar_full + 8 * q, 2 * kPartBytes);
+          tma_load_3d(smem_base + kLoadA[q] * kPartBytes, &map_q, bar_full + 8 * q, 64 * half, R0, kLoadA[q] * a.Hq + h);
+          tma_load_3d(smem_base + (3 + kLoadB[q]) * kPartBytes, &map_k, bar_full + 8 * q, 64 * half, C0,
+                      kLoadB[q] * a.Hkv + kvh);
         }
       }
       __syncwarp();
-      ok = __all_sync(0xffffffffu, mbar_wait(bar_full, half, a.status));
-      if (!ok) break;
-      tc_fence_after();
-      if (leader) {
 #pragma unroll
-        for (int q = 0; q < 6; ++q) {
+      for (int q = 0; q < 6; ++q) {
+        if (q < 3 && ok) {  // pair q needs the parts behind barrier q (the later pairs reuse parts already here)
+          ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * q, half, a.status));
+          tc_fence_after();
+        }
+        if (ok && leader) {
           const uint32_t a_addr = smem_base + kPairs[q][0] * kPartBytes;
           const uint32_t b_addr = smem_base + (3 + kPairs[q][1]) * kPartBytes;
 #pragma unroll
@@ -254,6 +261,10 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             acc = 1u;
           }
         }
+        __syncwarp();
+      }
+      if (!ok) break;
+      if (leader) {
         tc_commit(half == 0 ? bar_half : bar_done);
       }
       __syncwarp();
