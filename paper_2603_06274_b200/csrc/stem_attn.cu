@@ -248,6 +248,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* r) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
+               "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -498,6 +503,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       if (!ok) break;
       tc_fence_after();
       const float inv_l = 1.f / l_run;
+      const bool o_al32 = ((uintptr_t)a.O & 31u) == 0u;  // rows are multiples of 256 bytes apart
       __nv_bfloat16* o_row = a.O + ((int64_t)(q_tok0 + m) * a.Hq + h) * kHeadDim;
 #pragma unroll
       for (int c = 0; c < kHeadDim / 32; ++c) {
@@ -511,14 +517,18 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           if (lane == 0) mbar_arrive(bar(Smem::o_free, X));
         }
         if (row_valid) {
+          uint32_t w[16];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 w;
-            w.x = pack_bf16(o[q * 8 + 0] * inv_l, o[q * 8 + 1] * inv_l);
-            w.y = pack_bf16(o[q * 8 + 2] * inv_l, o[q * 8 + 3] * inv_l);
-            w.z = pack_bf16(o[q * 8 + 4] * inv_l, o[q * 8 + 5] * inv_l);
-            w.w = pack_bf16(o[q * 8 + 6] * inv_l, o[q * 8 + 7] * inv_l);
-            *(uint4*)(o_row + c * 32 + q * 8) = w;
+          for (int q = 0; q < 16; ++q) w[q] = pack_bf16(o[2 * q] * inv_l, o[2 * q + 1] * inv_l);
+          if (o_al32) {
+            // whole 32-byte sectors per store: a thread writes its own 256-byte row, so the stores of
+            // a warp are 32 separate sectors either way, and this halves their number
+            st_global_v8(o_row + c * 32, w);
+            st_global_v8(o_row + c * 32 + 16, w + 8);
+          } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+              *(uint4*)(o_row + c * 32 + q * 8) = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
           }
         }
       }
