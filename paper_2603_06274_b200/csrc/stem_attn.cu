@@ -48,7 +48,7 @@ constexpr int kCmdSlots = 4;
 constexpr int kOCol = 256;                               // O of slot X at kOCol + 128 X; S/P at 128 X
 constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;  // per wait
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
-constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // launch: 384 x 168; after: 256 x 208 + 128 x 88
+constexpr int kRegsSoftmax = 216, kRegsOther = 72;  // launch: 384 x 168; after: 256 x 216 + 128 x 72
 
 enum Role : int { kRoleSoftmax = 1, kRoleProducer = 2, kRoleMma = 3, kRoleQProducer = 4 };
 enum BarId : int { kBarKvFull = 1, kBarKvEmpty, kBarQFull, kBarQEmpty, kBarSFull, kBarPReady, kBarOFull, kBarOFree,
@@ -403,12 +403,27 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     uint32_t blk = 0;   // blocks of this slot so far (phase of s_full / p_ready)
     uint32_t ord = 0;   // non-empty items of this slot so far (phase of o_full / o_free)
     bool ok = true;
-    for (int item = (int)blockIdx.x + X * (int)gridDim.x; item < a.n_items && ok; item += 2 * (int)gridDim.x) {
+    // The list length of an item and whether its list ends on the diagonal block sit at the end of a
+    // chain of dependent global loads (work order -> row table -> length -> last entry).  The chain
+    // of the next item is walked while the current item's blocks are processed, and its result kept
+    // in one register (length, bit 31 = diagonal); the item's other fields are then cache hits.
+    auto list_info = [&](const int item) -> uint32_t {
+      if (item >= a.n_items) return 0u;
       const int h = a.work[2 * item], R = a.work[2 * item + 1];
       const int r = a.rows.row_r[R];
+      if (dense) return (uint32_t)(r + 1) | 0x80000000u;
+      const int n = min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max);
+      const bool diag = n > 0 && a.sel_idx[((int64_t)h * a.R_tot + R) * a.k_max + n - 1] >= r;
+      return (uint32_t)n | (diag ? 0x80000000u : 0u);
+    };
+    uint32_t next_info = list_info((int)blockIdx.x + X * (int)gridDim.x);
+    for (int item = (int)blockIdx.x + X * (int)gridDim.x; item < a.n_items && ok; item += 2 * (int)gridDim.x) {
+      const uint32_t info = next_info;
+      next_info = list_info(item + 2 * (int)gridDim.x);
+      const int h = a.work[2 * item], R = a.work[2 * item + 1];
       const int q_tok0 = a.rows.row_tok0[R];
       const int ntok = a.rows.row_ntok[R];
-      const int n = dense ? r + 1 : min(max(a.sel_cnt[(int64_t)h * a.R_tot + R], 0), a.k_max);
+      const int n = (int)(info & 0x7fffffffu);
       const bool row_valid = m < ntok;
       if (n == 0) {
         if (row_valid) {
@@ -419,7 +434,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         continue;
       }
-      const bool has_diag = dense || (a.sel_idx[((int64_t)h * a.R_tot + R) * a.k_max + n - 1] >= r);
+      const bool has_diag = (info >> 31) != 0u;
       float m_run = -INFINITY, l_run = 0.f;
       for (int e = 0; e < n; ++e, ++blk) {
         // S of block e is complete; so is every earlier tensor-core operation of this slot,
