@@ -11,9 +11,10 @@
 // terms are below 2^-24 of the leading one.  A pooled value that is not finite makes its row or
 // column of M NaN (which ranks below every number).
 //
-// One CTA per (128 x 128 tile of one sequence's causal triangle, query head), two CTAs per SM: TMA
-// brings the 3 + 3 operand parts (K-major, 128-byte swizzle) one half of the head dimension at a
-// time, one thread issues the 2 x 24 MMAs, the four warps
+// One CTA per (128 x 128 tile of one sequence's causal triangle, kv head): the Kbar parts stay in
+// shared memory while the Qbar parts of the group's query heads stream through (TMA, K-major,
+// 128-byte swizzle, one half of the head dimension per buffer); one warp issues the copies and the
+// 2 x 24 MMAs per head into one of two accumulators, the other four warps
 // read the accumulator (one row per thread), apply scale and bias, and either turn the tile through
 // shared memory and write the causal part of it with coalesced stores (the public M), or write each
 // row's selection keys as bit planes, one 128-byte line per 32 columns (the fused path's workspace
@@ -27,16 +28,19 @@ namespace stem {
 
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 288;                         // warps 0-7: epilogue (two warps per 32 accumulator rows, two 32-column
+                                                      // pieces each); warp 8: copies + MMAs
 constexpr int kTile = 128;
 constexpr int kPartBytes = kTile * 128;               // one operand part, one 64-column half of d (bf16): 16 KB
-constexpr int kSmemOps = 6 * kPartBytes;              // A hi/mid/lo, B hi/mid/lo (reused for both halves of d)
-constexpr int kSmemBias = kSmemOps;                   // 128 floats
-constexpr int kSmemBars = kSmemBias + kTile * 4;      // full[3], half_done, done
-constexpr int kSmemTmem = kSmemBars + 48;
+constexpr int kSmemB = 0;                             // Kbar parts, both halves: [half][part], resident for the whole CTA
+constexpr int kSmemA = kSmemB + 6 * kPartBytes;       // Qbar parts of one head: [half][part], refilled head by head
+constexpr int kSmemStage = kSmemA + 6 * kPartBytes;   // 8 warps x 32 rows x 32 columns fp32 (float output only)
+constexpr int kSmemBias = kSmemStage + 8 * 32 * 32 * 4;  // 128 floats
+constexpr int kSmemBars = kSmemBias + kTile * 4;      // b_full, a_full[2], a_empty[2], acc_full[2], acc_empty[2]
+constexpr int kSmemTmem = kSmemBars + 9 * 8;
 constexpr int kSmemTotal = kSmemTmem + 16;
-constexpr int kSmemBytes = kSmemTotal + 1024;         // slack for manual 1024-byte alignment; two CTAs per SM
-static_assert(kTile * kTile * 4 <= kSmemOps, "the output tile is staged over the operand tiles");
+constexpr int kSmemBytes = kSmemTotal + 1024;         // slack for manual 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 constexpr uint64_t kWaitLimitNs = 200ull * 1000 * 1000;
 
 __device__ __forceinline__ uint64_t globaltimer() {
@@ -46,6 +50,9 @@ __device__ __forceinline__ uint64_t globaltimer() {
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -130,14 +137,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both K-major, M = N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 
-// Monotone map float -> uint32 with -0 == +0 and NaN below everything (as -inf); every key is >= 1.
-__device__ __forceinline__ uint32_t metric_key(float f) {
-  uint32_t u = __float_as_uint(f);
-  if ((u & 0x7fffffffu) > 0x7f800000u) u = 0xff800000u;  // NaN -> -inf
-  if (u == 0x80000000u) u = 0u;                          // -0 -> +0
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-
 // In-register transpose of a 32 x 32 bit matrix: afterwards bit t of w[b] is bit b of the old w[t].
 __device__ __forceinline__ void transpose32(uint32_t (&w)[32]) {
 #pragma unroll
@@ -179,32 +178,38 @@ struct GemmArgs {
   int as_keys;  // write bit planes of the metric's selection keys (for launch_select_planes) instead of floats
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const GemmArgs a) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = ((uint32_t)__cvta_generic_to_shared(smem_raw) + 1023u) & ~1023u;
   unsigned char* smem_gen = smem_raw + (smem_base - (uint32_t)__cvta_generic_to_shared(smem_raw));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t bar_full = smem_base + kSmemBars, bar_half = bar_full + 24, bar_done = bar_full + 32;  // bar_full: 3 barriers
+  const uint32_t bars = smem_base + kSmemBars;
+  const uint32_t b_full = bars, a_full = bars + 8, a_empty = bars + 24, acc_full = bars + 40, acc_empty = bars + 56;
   float* bias = (float*)(smem_gen + kSmemBias);
 
+  // One CTA works on one tile of one sequence's causal triangle for the g query heads of a kv head:
+  // the Kbar parts stay in shared memory, the Qbar parts of the heads stream through, and two
+  // accumulators in tensor memory let the epilogue of one head overlap the MMAs of the next.
   const int seq = a.tiles[3 * blockIdx.x], ti = a.tiles[3 * blockIdx.x + 1], tj = a.tiles[3 * blockIdx.x + 2];
-  const int h = blockIdx.y, kvh = h / a.g;
+  const int kvh = blockIdx.y, g = a.g;
   const int nb = a.rows.seq_nblk[seq];
   const int row_off = a.rows.seq_row_off[seq];
   const int R0 = row_off + ti * kTile, C0 = row_off + tj * kTile;  // first global block row of A and of B
 
   if (threadIdx.x == 0) {
-    mbar_init(bar_full, 1);
-    mbar_init(bar_full + 8, 1);
-    mbar_init(bar_full + 16, 1);
-    mbar_init(bar_half, 1);
-    mbar_init(bar_done, 1);
+    mbar_init(b_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(a_full + 8 * i, 1);
+      mbar_init(a_empty + 8 * i, 1);
+      mbar_init(acc_full + 8 * i, 1);
+      mbar_init(acc_empty + 8 * i, 8);  // one arrival per epilogue warp
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + kSmemTmem), "n"(128)
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_base + kSmemTmem), "n"(256)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -212,8 +217,8 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   // its outputs are read only below this point.  (Without that launch attribute both are no-ops.)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  {
-    const int c = threadIdx.x;  // bias of column c of the tile
+  if (threadIdx.x < kTile) {
+    const int c = threadIdx.x;  // bias of column c of the tile (the same for every head of the group)
     bias[c] = (tj * kTile + c < nb) ? a.beta * a.mv[(int64_t)kvh * a.R_tot + C0 + c] : 0.f;
   }
   tc_fence_before();
@@ -221,130 +226,143 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = *(volatile uint32_t*)(smem_gen + kSmemTmem);
 
-  bool ok = true;
-  if (warp == 0) {
-    // The head dimension goes through shared memory in two halves of 64 columns (six 16 KB parts
-    // each), so that two CTAs fit on an SM and one's copies overlap the other's MMAs and epilogue.
+  if (warp == 8) {
+    // ============================== copies and MMAs ==============================
     const bool leader = elect_one();
+    bool ok = true;
+    auto load_a = [&](const int hh, const int half) {  // the three Qbar parts of one head, one half of d
+      if (leader) {
+        mbar_expect_tx(a_full + 8 * half, 3 * kPartBytes);
+#pragma unroll
+        for (int s = 0; s < 3; ++s)
+          tma_load_3d(smem_base + kSmemA + (half * 3 + s) * kPartBytes, &map_q, a_full + 8 * half, 64 * half, R0,
+                      s * a.Hq + kvh * g + hh);
+      }
+      __syncwarp();
+    };
+    if (leader) {
+      mbar_expect_tx(b_full, 6 * kPartBytes);
+#pragma unroll
+      for (int half = 0; half < 2; ++half)
+#pragma unroll
+        for (int s = 0; s < 3; ++s)
+          tma_load_3d(smem_base + kSmemB + (half * 3 + s) * kPartBytes, &map_k, b_full, 64 * half, C0, s * a.Hkv + kvh);
+    }
+    __syncwarp();
+    load_a(0, 0);
+    load_a(0, 1);
     // parts of A x parts of B, smallest products first: (mid,mid) (hi,lo) (lo,hi) (hi,mid) (mid,hi) (hi,hi)
     constexpr int kPairs[6][2] = {{1, 1}, {0, 2}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};
-    uint32_t acc = 0u;
 #pragma unroll 1
-    for (int half = 0; half < 2 && ok; ++half) {
-      if (half == 1) ok = __all_sync(0xffffffffu, mbar_wait(bar_half, 0, a.status));  // the first half's MMAs have read the parts
+    for (int st = 0; st < 2 * g; ++st) {
+      const int hh = st >> 1, half = st & 1;
+      const uint32_t acc_tmem = tmem + (uint32_t)(hh & 1) * 128u;
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(a_full + 8 * half, hh & 1, a.status));
+      if (ok && st == 0) ok = __all_sync(0xffffffffu, mbar_wait(b_full, 0, a.status));
+      // the accumulator was last used by head hh - 2: its epilogue must have read it
+      if (ok && half == 0 && hh >= 2) ok = __all_sync(0xffffffffu, mbar_wait(acc_empty + 8 * (hh & 1), ((hh >> 1) - 1) & 1, a.status));
       if (!ok) break;
-      // The copies go out in the order the products need them, two parts per barrier, so that the
-      // MMAs start when the first third of the bytes has landed.
-      constexpr int kLoadA[3] = {1, 0, 2}, kLoadB[3] = {1, 2, 0};
+      tc_fence_after();
       if (leader) {
+        uint32_t accf = half;  // the first MMA of a head overwrites the accumulator
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
-          mbar_expect_tx(bar_full + 8 * q, 2 * kPartBytes);
-          tma_load_3d(smem_base + kLoadA[q] * kPartBytes, &map_q, bar_full + 8 * q, 64 * half, R0, kLoadA[q] * a.Hq + h);
-          tma_load_3d(smem_base + (3 + kLoadB[q]) * kPartBytes, &map_k, bar_full + 8 * q, 64 * half, C0,
-                      kLoadB[q] * a.Hkv + kvh);
-        }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int q = 0; q < 6; ++q) {
-        if (q < 3 && ok) {  // pair q needs the parts behind barrier q (the later pairs reuse parts already here)
-          ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * q, half, a.status));
-          tc_fence_after();
-        }
-        if (ok && leader) {
-          const uint32_t a_addr = smem_base + kPairs[q][0] * kPartBytes;
-          const uint32_t b_addr = smem_base + (3 + kPairs[q][1]) * kPartBytes;
+        for (int q = 0; q < 6; ++q) {
+          const uint32_t a_addr = smem_base + kSmemA + (half * 3 + kPairs[q][0]) * kPartBytes;
+          const uint32_t b_addr = smem_base + kSmemB + (half * 3 + kPairs[q][1]) * kPartBytes;
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            mma_ss(tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), kIdesc, acc);
-            acc = 1u;
+            mma_ss(acc_tmem, smem_desc(a_addr + k * 32), smem_desc(b_addr + k * 32), kIdesc, accf);
+            accf = 1u;
           }
         }
-        __syncwarp();
-      }
-      if (!ok) break;
-      if (leader) {
-        tc_commit(half == 0 ? bar_half : bar_done);
+        tc_commit(a_empty + 8 * half);
+        if (half == 1) tc_commit(acc_full + 8 * (hh & 1));
       }
       __syncwarp();
-    }
-  }
-  // ---- epilogue: accumulator -> scale and bias -> shared memory (rows swizzled by 16-byte chunks)
-  ok = mbar_wait(bar_done, 0, a.status) && ok;
-  ok = __syncthreads_and(ok);
-  float* stage = (float*)smem_gen;  // 128 x 128 fp32 over the operand tiles, which are no longer needed
-  if (ok && a.as_keys) {
-    // For the selection: each thread turns the keys of its row, 32 columns at a time, into 32 bit
-    // planes (word k = bit k of the 32 keys) and stores them as one 128-byte line of the row.
-    tc_fence_after();
-    const int m = warp * 32 + lane;
-    const int r = ti * kTile + m;
-    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
-    const int stride = (nb + 31) & ~31;
-    uint32_t* dst = (uint32_t*)a.M + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)r * stride + tj * kTile;
-#pragma unroll 1
-    for (int gq = 0; gq < 4; ++gq) {
-      float v[32];
-      tmem_ld32(taddr + gq * 32, v);
-      tmem_ld_wait();
-      // key = bits ^ (negative ? all ones : sign bit) of the value with -0 -> +0 and NaN -> -inf; the
-      // exclusive-or is applied to the planes (32 operations for 32 keys) instead of to the keys
-      uint32_t w[32];
-#pragma unroll
-      for (int c = 0; c < 32; ++c)
-        w[c] = __float_as_uint(fmaxf(fmaf(a.scale, v[c], bias[gq * 32 + c]) + 0.0f, __int_as_float(0xff800000)));
-      transpose32(w);
-      const uint32_t neg = w[31];  // bit t: value t is negative
-#pragma unroll
-      for (int k = 0; k < 31; ++k) w[k] ^= neg;
-      w[31] = ~neg;
-      if (r < nb && tj * kTile + gq * 32 < stride) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q)
-          *(uint4*)(dst + gq * 32 + q * 4) = make_uint4(w[q * 4], w[q * 4 + 1], w[q * 4 + 2], w[q * 4 + 3]);
+      if (hh + 1 < g) {  // refill this half's buffer with the next head's parts once the MMAs have read it
+        ok = __all_sync(0xffffffffu, mbar_wait(a_empty + 8 * half, hh & 1, a.status));
+        if (!ok) break;
+        load_a(hh + 1, half);
       }
     }
-  } else if (ok) {
-    tc_fence_after();
-    const int m = warp * 32 + lane;  // row of the tile == TMEM lane
-    const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+  } else {
+    // ============================== epilogue ==============================
+    // A single warp per scheduler cannot keep the integer pipe busy (dependent chains), so two warps
+    // share each quarter of the accumulator rows: warps 0-3 take columns 0-63, warps 4-7 columns 64-127.
+    const int quarter = warp & 3, gq0 = (warp >> 2) * 2;
+    const int m = quarter * 32 + lane;  // row of the tile == TMEM lane
+    const int r = ti * kTile + m;       // row inside the sequence
+    const int stride = (nb + 31) & ~31;
+    float* stage = (float*)(smem_gen + kSmemStage) + warp * 32 * 32;
+    bool ok = true;
+#pragma unroll 1
+    for (int hh = 0; hh < g && ok; ++hh) {
+      const int h = kvh * g + hh;
+      ok = __all_sync(0xffffffffu, mbar_wait(acc_full + 8 * (hh & 1), (hh >> 1) & 1, a.status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t taddr = tmem + (uint32_t)(hh & 1) * 128u + ((uint32_t)(quarter * 32) << 16);
+      uint32_t* dst_planes = (uint32_t*)a.M + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)r * stride + tj * kTile;
+      float* mseq = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq];
+#pragma unroll 1
+      for (int gq = gq0; gq < gq0 + 2; ++gq) {
+        float v[32];
+        tmem_ld32(taddr + gq * 32, v);
+        tmem_ld_wait();
+        if (gq == gq0 + 1) {
+          // the accumulator is in registers: the MMAs of head hh + 2 may overwrite it
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty + 8 * (hh & 1));
+        }
+        if (a.as_keys) {
+          // For the selection: the keys of the row, 32 columns at a time, as 32 bit planes (word k =
+          // bit k of the 32 keys), one 128-byte line of the row.  key = bits ^ (negative ? all ones :
+          // sign bit) of the value with -0 -> +0 and NaN -> -inf; the exclusive-or is applied to the
+          // planes (32 operations for 32 keys) instead of to the keys.
+          uint32_t w[32];
 #pragma unroll
-    for (int gq = 0; gq < 4; ++gq) {
-      float v[32];
-      tmem_ld32(taddr + gq * 32, v);
-      tmem_ld_wait();
+          for (int c = 0; c < 32; ++c)
+            w[c] = __float_as_uint(fmaxf(fmaf(a.scale, v[c], bias[gq * 32 + c]) + 0.0f, __int_as_float(0xff800000)));
+          transpose32(w);
+          const uint32_t neg = w[31];  // bit t: value t is negative
 #pragma unroll
-      for (int c4 = 0; c4 < 8; ++c4) {
-        const int c = gq * 32 + c4 * 4;
-        float4 o;
-        o.x = fmaf(a.scale, v[c4 * 4 + 0], bias[c + 0]);
-        o.y = fmaf(a.scale, v[c4 * 4 + 1], bias[c + 1]);
-        o.z = fmaf(a.scale, v[c4 * 4 + 2], bias[c + 2]);
-        o.w = fmaf(a.scale, v[c4 * 4 + 3], bias[c + 3]);
-        *(float4*)(stage + m * kTile + (((c >> 2) ^ (m & 31)) << 2)) = o;
+          for (int k = 0; k < 31; ++k) w[k] ^= neg;
+          w[31] = ~neg;
+          if (r < nb && tj * kTile + gq * 32 < stride) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *(uint4*)(dst_planes + gq * 32 + q * 4) = make_uint4(w[q * 4], w[q * 4 + 1], w[q * 4 + 2], w[q * 4 + 3]);
+          }
+        } else {
+          // The public M: the warp's 32 x 32 piece through shared memory (rows swizzled by 16-byte
+          // chunks), then one 128-byte store per row, causal part only.
+#pragma unroll
+          for (int c4 = 0; c4 < 8; ++c4) {
+            float4 o;
+            o.x = fmaf(a.scale, v[c4 * 4 + 0], bias[gq * 32 + c4 * 4 + 0]);
+            o.y = fmaf(a.scale, v[c4 * 4 + 1], bias[gq * 32 + c4 * 4 + 1]);
+            o.z = fmaf(a.scale, v[c4 * 4 + 2], bias[gq * 32 + c4 * 4 + 2]);
+            o.w = fmaf(a.scale, v[c4 * 4 + 3], bias[gq * 32 + c4 * 4 + 3]);
+            *(float4*)(stage + lane * 32 + ((c4 ^ (lane & 7)) << 2)) = o;
+          }
+          __syncwarp();
+          const int cg = tj * kTile + gq * 32 + lane;  // this lane's column inside the sequence
+          for (int mm = 0; mm < 32; ++mm) {
+            const int rr = ti * kTile + quarter * 32 + mm;
+            if (rr >= nb) break;
+            if (cg <= rr) mseq[(int64_t)rr * nb + cg] = stage[mm * 32 + (((lane >> 2) ^ (mm & 7)) << 2) + (lane & 3)];
+          }
+          __syncwarp();
+        }
       }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 8) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(128) : "memory");
-  }
-  if (!ok || a.as_keys) return;
-  // ---- causal part of the tile to M, one row per step of a warp, 128 contiguous bytes per store
-  float* mseq = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq];
-  for (int mm = 0; mm < 32; ++mm) {
-    const int m = warp * 32 + mm;
-    const int r = ti * kTile + m;  // row inside the sequence
-    if (r >= nb) break;
-    float* dst = mseq + (int64_t)r * nb + tj * kTile;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int c = lane + 32 * q;
-      if (tj * kTile + c <= r) dst[c] = stage[m * kTile + (((c >> 2) ^ (m & 31)) << 2) + (c & 3)];
-    }
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(256) : "memory");
   }
 }
 
@@ -401,7 +419,7 @@ cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ks
     attr_set[dev_slot] = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)p.n_gemm_tiles, (unsigned)a.Hq);
+  cfg.gridDim = dim3((unsigned)p.n_gemm_tiles, (unsigned)a.Hkv);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = s;
