@@ -29,6 +29,11 @@
  *     returns STEM_ERR_INVALID_ARG / UNSUPPORTED / WORKSPACE.
  *   - Device-side waits are bounded; a wait that gives up records a code in the workspace,
  *     the kernel returns early, and stem_check_status reports STEM_ERR_DEVICE_TIMEOUT.
+ *   - Workspace: caller memory of stem_plan_info.workspace_bytes, 256-byte aligned.  Its first 32
+ *     bytes are the status words: they must be ZERO before the first hot call that uses the
+ *     workspace (cudaMemset them once after allocating); afterwards the library keeps them
+ *     (each kernel clears its own words when it is enqueued, stem_check_status clears all of them
+ *     after reporting a time-out).  The rest needs no initialisation.
  */
 #ifndef STEM_H_
 #define STEM_H_
@@ -115,7 +120,7 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
                size_t workspace_bytes, void* stream);
 
 /* stem_score for callers that cannot hand the library a workspace.  (The paper has no counterpart;
- * this is a packaging variant of stem_score, computing the same M.)
+ * this is a packaging variant of stem_score: same two kernels, same M.)
  *
  * Who needs it: code that runs where device allocation is off limits - a plug-in called from inside
  * a serving engine whose memory pool already owns the whole GPU, a callback that must not touch the
@@ -128,19 +133,23 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
  * cudaMalloc / cudaFree and uses no allocating routine; the plan must have been created earlier
  * (plan creation does allocate its small tables).
  *
- *   - M is required.  Same layout and values as stem_score with a workspace.
- *   - Problems whose pooled tensors exceed the array, i.e.
- *       (H_q * R_tot + H_kv * W) * 128 * 4 + H_kv * R_tot * 4 bytes (each part rounded up to 256),
- *       W = sum over the sequences of N_blk rounded up to a multiple of 64,
+ *   - M is required.  Same layout as stem_score with a workspace, and the same values (the same
+ *     pooling and metric kernels run on the same inputs).
+ *   - Problems whose status words and pooled tensors exceed the array, i.e.
+ *       256 + H_kv * R_tot * 4 + (H_q + H_kv) * R_tot * 128 * 6 bytes (each part rounded up to 256)
  *       > STEM_STATIC_SCRATCH_BYTES,
  *     are rejected with STEM_ERR_STATIC_SCRATCH and nothing is enqueued.
  *   - The first call on each device resolves the array's device address (a one-time set-up that
  *     talks to the CUDA runtime); make that first call before starting any stream capture.  The
  *     plan's device must be the current device.
  *   - All calls on a device share the one array.  Its contents are whatever the previous call
- *     left; every element this call reads it has written first, so nothing needs clearing.  Two
- *     calls that overlap on the GPU (different streams, no ordering between them) race on the
- *     array: serialise them. */
+ *     left: the call clears the status words it needs at zero, and overwrites every pooled element
+ *     its result depends on before reading it (metric tiles that reach past a sequence's last
+ *     block do read stale rows, but only into entries that are never stored).  Two calls that
+ *     overlap on the GPU (different streams, no ordering between them) race on the array:
+ *     serialise them.
+ *   - A bounded wait that gave up inside this call is reported by stem_check_status called with
+ *     workspace == NULL. */
 #define STEM_STATIC_SCRATCH_BYTES (8u * 1024u * 1024u)
 int stem_score_static(const stem_plan* plan, const void* Q, const void* K, const void* V, float* M, void* stream);
 
@@ -154,8 +163,8 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
                 size_t workspace_bytes, void* stream);
 
 /* Alg. 1 steps 1-3c in one call: block-wise representations, Output-Aware Metric (Eq. 7), Token
- * Position-Decay budget (Eq. 3) and top-k selection; the metric is kept in the workspace
- *   (fp32 [num_q_heads, metric_elems], part of workspace_bytes), never handed to the caller.
+ * Position-Decay budget (Eq. 3) and top-k selection; the metric is kept in the workspace (as bit
+ *   planes of its order-preserving selection keys, part of workspace_bytes), never handed to the caller.
  *   Same results as stem_score(M = NULL) followed by stem_select(M = NULL).
  *   Writes sel_idx / sel_cnt; leaves the pooled tensors in the workspace. */
 int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const void* V, int32_t* sel_idx,
@@ -176,12 +185,20 @@ int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, con
 int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
                  int32_t* sel_cnt, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
-/* Synchronises `stream`, then reads and clears the device status words of `workspace`.
+/* Synchronises `stream`, then reads the device status words of `workspace` (workspace == NULL: of
+ * the scratch built into the library, see stem_score_static) and clears them if they are set.
  * Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in a kernel gave up; outputs of that
  * call are undefined) or STEM_ERR_CUDA.  detail (optional, HOST int32[4]) receives the raw words:
- * {code, block index, role, barrier id} of the attention kernel (code 1), or {2, tile, head, 0} when
+ * {1, CTA index, role, barrier id} of the attention kernel, or {2, tile, kv head, 0} when
  * the wait that gave up was in the metric kernel. */
 int stem_check_status(const stem_plan* plan, void* workspace, void* stream, int32_t* detail_host);
+
+/* Self-test of the time-out reporting (the paper has no counterpart).  Enqueues a one-thread kernel
+ * that waits 1 ms, with the same bounded-wait routine the attention and metric kernels use, on a
+ * barrier nothing ever arrives at, records {1, 0, 99, 0} in the workspace status words and returns
+ * normally.  A following stem_check_status must report STEM_ERR_DEVICE_TIMEOUT; the CUDA context
+ * stays usable.  Never needed in production. */
+int stem_selftest_wait_timeout(const stem_plan* plan, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Number of kernels the last hot call on this plan launched (for launch accounting). */
 int stem_last_launch_count(const stem_plan* plan);

@@ -25,7 +25,7 @@ STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_destroy", "stem_plan_query",
            "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_score_select", "stem_sparse_prefill", "stem_prefill",
-           "stem_check_status", "stem_last_launch_count")
+           "stem_check_status", "stem_selftest_wait_timeout", "stem_last_launch_count")
 
 
 class StemConfig(ctypes.Structure):
@@ -106,6 +106,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_sparse_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_prefill.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_check_status.argtypes = [vp, vp, vp, i32p]
+    lib.stem_selftest_wait_timeout.argtypes = [vp, vp, ctypes.c_size_t, vp]
     lib.stem_last_launch_count.argtypes = [vp]
     for name in EXPORTS:
         if name not in ("stem_status_string",):
@@ -254,9 +255,23 @@ def stem_prefill(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tens
                                _ptr(lse), p, n, _stream()), "stem_prefill")
 
 
-def stem_check_status(plan: StemPlan, workspace: Optional[torch.Tensor] = None):
-    """Synchronise the current stream and return (status, detail[4])."""
-    p, _ = _ws_args(plan, workspace)
+def stem_check_status(plan: StemPlan, workspace: Optional[torch.Tensor] = None, static_scratch: bool = False):
+    """Synchronise the current stream and return (status, detail[4]).  With ``static_scratch`` the status
+    words of the scratch built into the library (stem_score_static) are read instead of a workspace's."""
+    p = None if static_scratch else _ws_args(plan, workspace)[0]
     detail = (ctypes.c_int32 * 4)()
     st = load().stem_check_status(plan.handle, p, _stream(), ctypes.cast(detail, ctypes.POINTER(ctypes.c_int32)))
     return int(st), [int(x) for x in detail]
+
+
+def status_words(plan: StemPlan, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The eight int32 status words at the start of the (aligned) workspace, as a view."""
+    ws = plan.workspace() if workspace is None else workspace
+    off = (-ws.data_ptr()) % 256
+    return ws[off:off + 32].view(torch.int32)
+
+
+def stem_selftest_wait_timeout(plan: StemPlan, workspace: Optional[torch.Tensor] = None) -> None:
+    """Enqueue the library's time-out self-test: a 1 ms bounded wait that runs out and records it."""
+    p, n = _ws_args(plan, workspace)
+    _check(load().stem_selftest_wait_timeout(plan.handle, p, n, _stream()), "stem_selftest_wait_timeout")

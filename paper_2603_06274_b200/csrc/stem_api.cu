@@ -114,7 +114,6 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_len(batch), seq_nblk(batch),
       seq_row_off(batch);
   std::vector<int64_t> seq_m_off(batch), seq_mt_off(batch);
-  std::vector<int32_t> seq_kt_off(batch);
   int64_t m_off = 0, mt_off = 0;
   for (int b = 0; b < batch; ++b) {
     const int32_t n = p.cu[b + 1] - p.cu[b];
@@ -126,8 +125,6 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     seq_m_off[b] = m_off;
     seq_mt_off[b] = mt_off;
     mt_off += (int64_t)nb * ((nb + 31) / 32 * 32);  // rows padded to whole 32-column groups
-    seq_kt_off[b] = p.kt_width;
-    p.kt_width += (nb + 63) / 64 * 64;
     m_off += (int64_t)nb * nb;
     p.max_nblk = std::max(p.max_nblk, nb);
     const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb) / 1000;
@@ -155,33 +152,9 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.selected_pairs *= Hq;
   p.causal_pairs *= Hq;
 
-  // Score/select tiles: one CTA scores the g heads of a kv group for a run of consecutive rows.
-  // A tile holds at most 32 pooled query vectors and one candidate list per vector in shared
-  // memory, which bounds the vectors per tile when the budget (list length) is large.
-  if (p.max_nblk > score_select_max_blocks()) {
+  if (p.max_nblk > row_select_max_blocks()) {
     delete sp;
     return STEM_ERR_UNSUPPORTED;
-  }
-  const size_t list_bytes = score_select_list_bytes(p.k_max);
-  int nq_cap = 32;
-  while (nq_cap > g && (size_t)((nq_cap + 7) / 8 * 8) * list_bytes > score_select_smem_budget()) nq_cap /= 2;
-  if ((size_t)((std::max(1, nq_cap / g) * g + 7) / 8 * 8) * list_bytes > score_select_smem_budget()) {
-    delete sp;
-    return STEM_ERR_UNSUPPORTED;
-  }
-  p.sel_rows_per_tile = std::max(1, nq_cap / g);
-  p.sel_nq = p.sel_rows_per_tile * g;
-  std::vector<int32_t> tiles;
-  {
-    std::vector<std::pair<int32_t, std::pair<int32_t, int32_t>>> t;  // (last row, (seq, r0)), long rows first
-    for (int b = 0; b < batch; ++b)
-      for (int32_t r0 = 0; r0 < seq_nblk[b]; r0 += p.sel_rows_per_tile) t.push_back({r0, {b, r0}});
-    std::stable_sort(t.begin(), t.end(), [](auto& a, auto& b) { return a.first > b.first; });
-    for (auto& e : t) {
-      tiles.push_back(e.second.first);
-      tiles.push_back(e.second.second);
-    }
-    p.n_sel_tiles = (int32_t)t.size();
   }
 
   // Tiles of the metric GEMM: the 128 x 128 tiles of every sequence's causal triangle, long rows first.
@@ -239,8 +212,7 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
                o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
                o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
                o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off), o_seq_mt_off = push(blob, seq_mt_off),
-               o_seq_kt_off = push(blob, seq_kt_off),
-               o_tiles = push(blob, tiles), o_gt = push(blob, gemm_tiles), o_ws = push(blob, work_sparse),
+               o_gt = push(blob, gemm_tiles), o_ws = push(blob, work_sparse),
                o_wd = push(blob, work_dense);
   if (cudaMalloc(&p.d_blob, blob.size()) != cudaSuccess ||
       cudaMemcpy(p.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -261,8 +233,6 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
   p.rows.seq_mt_off = (const int64_t*)(d + o_seq_mt_off);
-  p.rows.seq_kt_off = (const int32_t*)(d + o_seq_kt_off);
-  p.d_sel_tiles = (const int32_t*)(d + o_tiles);
   p.d_gemm_tiles = (const int32_t*)(d + o_gt);
   p.d_work_sparse = (const int32_t*)(d + o_ws);
   p.d_work_dense = (const int32_t*)(d + o_wd);
@@ -339,7 +309,7 @@ static int enqueue_score_select(const Plan& p, const void* Q, const void* K, con
   float* M = (float*)(w + p.ws.metric);  // holds the bit planes of the selection keys, not the floats
   int rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, true, true, (int32_t*)(w + p.ws.status), s));
@@ -363,7 +333,7 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   float* mv = (float*)(w + p.ws.mv);
   rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, nullptr, nullptr, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   if (M) {
@@ -451,11 +421,22 @@ int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void
 }
 
 int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* detail) {
-  if (!plan || !ws) return STEM_ERR_INVALID_ARG;
+  if (!plan) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
   cudaStream_t s = (cudaStream_t)stream;
   int32_t words[kStatusWords] = {0};
-  uint8_t* w = (uint8_t*)ws + p.ws.status;
+  uint8_t* w = nullptr;
+  if (ws) {
+    w = (uint8_t*)ws + p.ws.status;
+  } else {
+    // no workspace: the status words of the scratch built into the library (stem_score_static)
+    int device = -1;
+    int32_t* st = nullptr;
+    if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+    const int rc = static_scratch_status_words(device, &st);
+    if (rc != STEM_OK) return rc;
+    w = (uint8_t*)st;
+  }
   if (cudaStreamSynchronize(s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   if (cudaMemcpy(words, w, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   if (detail) std::memcpy(detail, words, 4 * sizeof(int32_t));
@@ -465,6 +446,14 @@ int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* de
     return STEM_ERR_DEVICE_TIMEOUT;
   }
   return STEM_OK;
+}
+
+int stem_selftest_wait_timeout(const stem_plan* plan, void* ws, size_t ws_bytes, void* stream) {
+  if (!plan) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  const int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  return cuda_rc(launch_selftest_wait((int32_t*)((uint8_t*)ws + p.ws.status), (cudaStream_t)stream));
 }
 
 }  // extern "C"

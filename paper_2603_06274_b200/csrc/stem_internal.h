@@ -16,6 +16,7 @@ constexpr int kHeadDim = 128;
 //   [0] code (0 = ok, 1 = a bounded wait of the attention kernel gave up)   [1] CTA index   [2] role   [3] barrier id
 //   [4] code (2 = a bounded wait of the metric kernel gave up)   [5] tile   [6] head
 constexpr int kStatusWords = 8;
+constexpr int kRoleSelfTest = 99;  // role recorded by stem_selftest_wait_timeout
 
 // Device-side row tables, built once per plan.
 struct RowTables {
@@ -30,7 +31,6 @@ struct RowTables {
   const int32_t* seq_row_off;  // [batch] global row of the sequence's row 0
   const int64_t* seq_m_off;    // [batch] offset of the sequence's square inside one head of M
   const int64_t* seq_mt_off;   // [batch] offset of the sequence inside one head of the bit-plane metric
-  const int32_t* seq_kt_off;   // [batch] first column of the sequence inside a row of Kbar^T (multiple of 64)
 };
 
 // Where things live inside the caller's workspace (byte offsets, 256-aligned).
@@ -51,7 +51,6 @@ struct Plan {
   int device = 0;
   int sm_count = 0;
   int32_t T = 0, R_tot = 0, k_max = 0, max_nblk = 0;
-  int32_t kt_width = 0;  // row length of Kbar^T: sum over sequences of N_blk rounded up to 64
   int64_t m_tot = 0;
   int64_t mt_tot = 0;  // words per head of the bit-plane metric: sum_b N_blk(b) * roundup(N_blk(b), 32)
   int64_t selected_blocks = 0, causal_blocks = 0, selected_pairs = 0, causal_pairs = 0;
@@ -61,10 +60,6 @@ struct Plan {
   // device blob
   void* d_blob = nullptr;
   RowTables rows{};
-  const int32_t* d_sel_tiles = nullptr;  // [n_sel_tiles][2] (sequence, first row) of the score/select tiles
-  int32_t n_sel_tiles = 0;
-  int32_t sel_rows_per_tile = 0;         // rows of one tile (all heads of a kv group ride together)
-  int32_t sel_nq = 0;                    // pooled query vectors per tile
   const int32_t* d_gemm_tiles = nullptr;  // [n_gemm_tiles][3] (sequence, row tile, column tile) of the metric GEMM
   int32_t n_gemm_tiles = 0;
   const int32_t* d_work_sparse = nullptr;  // [n_items][2] (head, global row), attention work order
@@ -76,11 +71,9 @@ struct Plan {
 };
 
 // Kernel launchers (each returns the cudaError_t of the launch).
-// qbar: [H_q, R_tot, d]; kbar_t: [H_kv, d, kt_width] (transposed for the scoring GEMM); mv: [H_kv, R_tot].
-// qbar / kbar_t (optional, fp32) and qsplit / ksplit (optional, both or neither: bf16 [3, H, R_tot, d], the pooled
-// vectors as hi + mid + lo parts) are two forms of the same pooled vectors; a caller asks for the one it reads.
-cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t,
-                        float* mv, void* qsplit, void* ksplit, cudaStream_t s);
+// Alg. 1 step 1: mv fp32 [H_kv, R_tot]; qsplit / ksplit bf16 [3, H, R_tot, d], the pooled vectors as hi + mid + lo parts.
+cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* mv, void* qsplit, void* ksplit,
+                        cudaStream_t s);
 
 // Metric of every causal block (layout of stem_score's M) from the split pooled vectors, on the tensor cores.
 // as_keys: instead of the floats, store bit planes of the selection's order-preserving keys: row r of sequence b at
@@ -90,17 +83,6 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
 // kernel's tail).  The caller clears status words 4..7 beforehand.
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
                                bool as_keys, bool dependent, int32_t* status, cudaStream_t s);
-
-// Shared-memory needs of the score/select kernel, for sizing its tiles at plan creation.
-size_t score_select_list_bytes(int k_max);   // per pooled query vector
-size_t score_select_smem_budget();            // bytes available for the candidate lists of a tile
-int score_select_max_blocks();                // largest supported N_blk of a sequence
-
-// mode bits for launch_score_select
-enum : int { kFromPooled = 1, kFromMetric = 2, kWriteMetric = 4, kSelect = 8 };
-cudaError_t launch_score_select(const Plan& p, int mode, const float* qbar, const float* kbar_t, const float* mv,
-                                const float* M_in, float* M_out, int32_t* sel_idx, int32_t* sel_cnt,
-                                cudaStream_t s);
 
 // Selection from a stored metric (layout of stem_score's M), one warp per (head, row).
 int row_select_max_blocks();  // largest supported N_blk of a sequence
@@ -113,6 +95,12 @@ cudaError_t launch_select_planes(const Plan& p, const uint32_t* Mt, bool depende
 cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
                                     const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,
                                     int32_t* status, cudaStream_t s);
+
+// One thread waits 1 ms on a barrier nobody arrives at and records the time-out in status words 0..3.
+cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);
+
+// Status words of the scratch built into the library (stem_score_static) on the current device.
+int static_scratch_status_words(int device, int32_t** out);
 
 }  // namespace stem
 

@@ -35,10 +35,9 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
 template <int kBlock>
 __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                                                    const __nv_bfloat16* __restrict__ V, int64_t q_st, int64_t q_sh,
-                                                   int64_t kv_st, int64_t kv_sh, int Hq, int Hkv, int R_tot, int kt_width,
-                                                   RowTables rows, float* __restrict__ qbar, float* __restrict__ kbar_t,
-                                                   float* __restrict__ mv, __nv_bfloat16* __restrict__ qsplit,
-                                                   __nv_bfloat16* __restrict__ ksplit) {
+                                                   int64_t kv_st, int64_t kv_sh, int Hq, int Hkv, int R_tot,
+                                                   RowTables rows, float* __restrict__ mv,
+                                                   __nv_bfloat16* __restrict__ qsplit, __nv_bfloat16* __restrict__ ksplit) {
   constexpr int kTokPerWarp = kBlock / 4;
   constexpr int kSteps = kTokPerWarp / 2;
   // lets a kernel launched as a programmatic dependent set itself up during this kernel's last wave
@@ -89,27 +88,18 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
     const int c = threadIdx.x;
     const float sum = (red[0][c] + red[1][c]) + (red[2][c] + red[3][c]);
     const float mean = sum / (float)ntok;
-    if (qsplit != nullptr) {
-      // mean = hi + mid + lo, each part the bf16 rounding of what the previous ones leave (the tensor-core
-      // metric kernel multiplies these parts); row = global block row for both tensors
-      const __nv_bfloat16 hi = __float2bfloat16_rn(mean);
-      const float r1 = mean - __bfloat162float(hi);
-      const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-      const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-      __nv_bfloat16* dst = kind == 0 ? qsplit : ksplit;
-      const int64_t plane = (int64_t)(kind == 0 ? Hq : Hkv) * R_tot * kHeadDim;
-      const int64_t at = ((int64_t)h * R_tot + R) * kHeadDim + c;
-      dst[at] = hi;
-      dst[at + plane] = mid;
-      dst[at + 2 * plane] = lo;
-    }
-    if (kind == 0) {
-      if (qbar != nullptr) qbar[((int64_t)h * R_tot + R) * kHeadDim + c] = mean;
-    } else if (kbar_t != nullptr) {
-      // Kbar is stored transposed ([H_kv, d, kt_width], block index contiguous) for the scoring GEMM
-      const int col = rows.seq_kt_off[rows.row_seq[R]] + rows.row_r[R];
-      kbar_t[((int64_t)h * kHeadDim + c) * kt_width + col] = mean;
-    }
+    // mean = hi + mid + lo, each part the bf16 rounding of what the previous ones leave (the tensor-core
+    // metric kernel multiplies these parts); row = global block row for both tensors
+    const __nv_bfloat16 hi = __float2bfloat16_rn(mean);
+    const float r1 = mean - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    __nv_bfloat16* dst = kind == 0 ? qsplit : ksplit;
+    const int64_t plane = (int64_t)(kind == 0 ? Hq : Hkv) * R_tot * kHeadDim;
+    const int64_t at = ((int64_t)h * R_tot + R) * kHeadDim + c;
+    dst[at] = hi;
+    dst[at + plane] = mid;
+    dst[at + 2 * plane] = lo;
   } else {
     float best = 0.f;  // squared norms are >= 0
 #pragma unroll
@@ -137,8 +127,8 @@ __global__ void __launch_bounds__(128) pool_kernel(const __nv_bfloat16* __restri
 
 }  // namespace
 
-cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* qbar, float* kbar_t, float* mv,
-                        void* qsplit, void* ksplit, cudaStream_t s) {
+cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* mv, void* qsplit, void* ksplit,
+                        cudaStream_t s) {
   const int slots = p.cfg.num_q_heads + 2 * p.cfg.num_kv_heads;
   const dim3 grid((unsigned)((int64_t)p.R_tot * slots));
   auto q = (const __nv_bfloat16*)Q;
@@ -146,12 +136,12 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
   auto v = (const __nv_bfloat16*)V;
   if (p.cfg.block == 128)
     pool_kernel<128><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
-                                          p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
-                                          p.rows, qbar, kbar_t, mv, (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
+                                          p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.rows, mv,
+                                          (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
   else
     pool_kernel<64><<<grid, 128, 0, s>>>(q, k, v, p.cfg.q_stride_tok, p.cfg.q_stride_head, p.cfg.kv_stride_tok,
-                                         p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.kt_width,
-                                         p.rows, qbar, kbar_t, mv, (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
+                                         p.cfg.kv_stride_head, p.cfg.num_q_heads, p.cfg.num_kv_heads, p.R_tot, p.rows, mv,
+                                         (__nv_bfloat16*)qsplit, (__nv_bfloat16*)ksplit);
   return cudaGetLastError();
 }
 

@@ -18,6 +18,7 @@
 #include <cuda_runtime.h>
 
 #include "stem_internal.h"
+#include "stem_ptx.cuh"
 
 namespace stem {
 
@@ -33,34 +34,7 @@ __device__ __forceinline__ uint32_t metric_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// In-register transpose of a 32 x 32 bit matrix: afterwards bit t of w[b] is bit b of the old w[t].
-__device__ __forceinline__ void transpose32(uint32_t (&w)[32]) {
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {  // 16-bit halves: byte permutes
-    const uint32_t lo = __byte_perm(w[k], w[k + 16], 0x5410), hi = __byte_perm(w[k], w[k + 16], 0x7632);
-    w[k] = lo;
-    w[k + 16] = hi;
-  }
-#pragma unroll
-  for (int k = 0; k < 32; ++k) {  // bytes
-    if (k & 8) continue;
-    const uint32_t lo = __byte_perm(w[k], w[k + 8], 0x6240), hi = __byte_perm(w[k], w[k + 8], 0x7351);
-    w[k] = lo;
-    w[k + 8] = hi;
-  }
-#pragma unroll
-  for (int s = 2; s < 5; ++s) {
-    const int j = 16 >> s;
-    const uint32_t mhi = s == 2 ? 0xf0f0f0f0u : s == 3 ? 0xccccccccu : 0xaaaaaaaau;
-#pragma unroll
-    for (int k = 0; k < 32; ++k) {
-      if (k & j) continue;
-      const uint32_t x = w[k], y = w[k + j];
-      w[k] = (x & ~mhi) | ((y << j) & mhi);
-      w[k + j] = ((x >> j) & ~mhi) | (y & mhi);
-    }
-  }
-}
+using ptx::transpose32;
 
 struct SelArgs {
   const float* M;

@@ -47,6 +47,8 @@ class Workload:
     # input recipe switches
     heavy_mode: str = "bernoulli"   # "bernoulli": K row 0 + 2% of rows x4; "window": 8 rows per 4096-token window x4
     sink: bool = False              # add a shared direction to the first 4 K rows and to every Q row
+    v_recipe: str = "norm_lognormal"  # "norm_lognormal": ||V_t|| itself is log-normal(0, 0.5) (elements ~ 0.1);
+                                      # "gain_lognormal": V_t = g_t z_t with z_t ~ N(0, I), elements O(1)
     seed: int = BASE_SEED
     layers: int = 1
 
@@ -131,7 +133,9 @@ def make_qkv(w: Workload, layer: int = 0) -> Dict[str, np.ndarray]:
     Recipe: Q, K i.i.d. N(0,1).  V_t = g_t * z_t / ||z_t|| with z_t ~ N(0, I) and
     g_t = exp(0.5 n_t), n_t ~ N(0,1), per token and kv head, i.e. the per-token value norm is
     log-normal(0, 0.5): about half of the tokens have ||V_t|| < 1, so the max(0, .) clamp of the
-    magnitude term is exercised, and block maxima of ln ||V|| are O(1).  A sparse set of K
+    magnitude term is exercised, and block maxima of ln ||V|| are O(1).  With
+    ``v_recipe = "gain_lognormal"`` the normalisation is left out (V_t = g_t z_t: elements of
+    order one, norms about sqrt(d) times larger, outputs about sqrt(d) times larger).  A sparse set of K
     rows per kv head is scaled by 4 ("heavy" keys): either row 0 of each sequence plus a
     Bernoulli(0.02) subset, or 8 uniformly placed rows in every 4096-token window.  With
     ``sink`` a unit direction u per kv head is added (x8) to the first 4 K rows of each
@@ -160,7 +164,12 @@ def make_qkv(w: Workload, layer: int = 0) -> Dict[str, np.ndarray]:
         kc = rk.standard_normal((n, hkv, d), dtype=np.float32)
         vc = rv.standard_normal((n, hkv, d), dtype=np.float32)
         gain = np.exp(0.5 * rn.standard_normal((n, hkv, 1), dtype=np.float32))
-        vc *= gain / np.linalg.norm(vc, axis=2, keepdims=True)
+        if w.v_recipe == "norm_lognormal":
+            vc *= gain / np.linalg.norm(vc, axis=2, keepdims=True)
+        elif w.v_recipe == "gain_lognormal":
+            vc *= gain
+        else:
+            raise ValueError(w.v_recipe)
         # heavy keys
         if w.heavy_mode == "bernoulli":
             heavy = rh.random((n, hkv)) < 0.02

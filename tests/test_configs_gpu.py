@@ -1,11 +1,13 @@
-"""GPU parity at the full sizes of the five benchmark configurations, in the launch configuration
-bench.py times (the fused stem_prefill call).
+"""GPU parity at the full sizes of the five benchmark configurations and their sweeps, in the launch
+configuration bench.py times (the fused stem_prefill call).
 
 Scoring and selection are compared with the CPU checker for EVERY (head, row): list lengths must
 equal the budget table, lists must be identical except at logged near-ties of the checker's metric
-(relative gap <= 1e-3 at the top-k boundary).  Attention is compared on a sample of (head, row)
-lists the checker can compute one by one: structural rows of every head (first, last of the dense
-triangle, first sparse, middle, last) plus seeded random rows, on the index lists the GPU used."""
+(relative gap <= 1e-3 at the top-k boundary).  Attention is compared, on the index lists the GPU
+used, for every list of the 4K and 32K configurations, for every list of the heads of kv group 0
+of the 128K configurations, and on a sample elsewhere: structural rows of every head (first, last
+of the dense triangle, first sparse, middle, last) plus seeded random rows.  Rows outside the
+comparison are checked to be finite."""
 import numpy as np
 import pytest
 import torch
@@ -17,14 +19,20 @@ from tests._util import check_attention, compare_selection, from_dev_bf16, oracl
 
 pytestmark = pytest.mark.gpu
 
+# (configuration, overrides, attention coverage): "all" = every list, "group0" = every list of the heads of
+# kv group 0 plus the sample, "sample" = the sample only
 CASES = [
-    ("cfg1", {}),
-    ("cfg2", {}),
-    ("cfg3", {}),
-    ("cfg4", {"budget_permille": 50}),
-    ("cfg4", {"budget_permille": 200}),
-    ("cfg5", {}),                           # the paper's schedule, mu = 7/10
-    ("cfg5", {"mu_num": 1, "mu_den": 1}),   # no decay
+    ("cfg1", {}, "all"),
+    ("cfg2", {}, "all"),
+    ("cfg3", {}, "group0"),
+    ("cfg4", {"budget_permille": 30}, "sample"),
+    ("cfg4", {"budget_permille": 50}, "group0"),
+    ("cfg4", {"budget_permille": 100}, "sample"),
+    ("cfg4", {"budget_permille": 200}, "sample"),
+    ("cfg5", {}, "group0"),                           # the paper's schedule, mu = 7/10
+    ("cfg5", {"mu_num": 1, "mu_den": 1}, "sample"),   # no decay
+    ("cfg5", {"mu_num": 1, "mu_den": 2}, "sample"),   # linear decay to half the budget
+    ("cfg5", {"stem_blocks": 4, "local_blocks": 4, "min_blocks": 54}, "sample"),  # forced blocks and minimum as printed
 ]
 
 _data_cache = {}
@@ -39,8 +47,9 @@ def _data(name):
     return _data_cache[name]
 
 
-@pytest.mark.parametrize("name,overrides", CASES, ids=[f"{n}-{'-'.join(f'{k}{v}' for k, v in o.items()) or 'base'}" for n, o in CASES])
-def test_full_size_config(name, overrides):
+@pytest.mark.parametrize("name,overrides,coverage", CASES,
+                         ids=[f"{n}-{'-'.join(f'{k}{v}' for k, v in o.items()) or 'base'}" for n, o, _ in CASES])
+def test_full_size_config(name, overrides, coverage):
     w = wl.CONFIGS[name].with_(**overrides)
     data, q, k, v = _data(name)
     plan = StemPlan.from_workload(w)
@@ -68,16 +77,21 @@ def test_full_size_config(name, overrides):
     assert len(ties) <= max(2, n_lists // 200)
     del M_ref
 
-    # ---- attention on sampled lists, given the GPU's index set
+    # ---- attention, given the GPU's index set
     k_s = [so.k_start(int(nb), p) for nb in nblk]
-    rows = sample_rows(w.num_q_heads, nblk, [k_s[0] - 1, k_s[0]], n_random=24, seed=w.seed)
+    g = w.num_q_heads // w.num_kv_heads
+    if coverage == "all":
+        rows = None
+    else:
+        rows = sample_rows(w.num_q_heads, nblk, [k_s[0] - 1, k_s[0]], n_random=24, seed=w.seed,
+                           full_heads=range(g) if coverage == "group0" else ())
     O_ref, _ = so.attention(data["q"], data["k"], data["v"], data["cu_seqlens"], w.block, idx_g, cnt_g, rows=rows,
                             want_lse=False)
     o_gpu = from_dev_bf16(out)
     mask = ~np.isnan(O_ref)
     assert mask.any()
-    mx, mean = check_attention(o_gpu, O_ref, mask)
-    print(f"{w.name}: attention on {len(rows)} sampled lists: max abs {mx:.3e}, mean abs {mean:.3e}")
+    n_cmp = n_lists if rows is None else len(rows)
+    check_attention(o_gpu, O_ref, mask, label=f"{w.name} {overrides or ''} ({n_cmp} of {n_lists} lists)")
     # every output row was written
     assert torch.isfinite(out.float()).all()
     plan.close()

@@ -92,3 +92,10 @@ def test_equal_metrics_are_broken_by_block_id_in_the_fused_path():
     n = int(cnt_g[1, r])
     want = np.concatenate([np.arange(0, n - w.local_blocks), np.arange(r + 1 - w.local_blocks, r + 1)])
     assert np.array_equal(idx_g[1, r, :n], want)
+
+
+def test_32k_layer_with_value_elements_of_order_one():
+    # the 32K configuration on the value recipe V_t = g_t z_t (elements O(1), outputs ~ sqrt(d) times larger)
+    w = wl.CONFIGS["cfg2"].with_(v_recipe="gain_lognormal", name="cfg2_gain_v")
+    data, q, k, v = _dev(w)
+    check_full_path(w, data, q, k, v, n_random=200)
