@@ -140,8 +140,10 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
  *       > STEM_STATIC_SCRATCH_BYTES,
  *     are rejected with STEM_ERR_STATIC_SCRATCH and nothing is enqueued.
  *   - The first call on each device resolves the array's device address (a one-time set-up that
- *     talks to the CUDA runtime); make that first call before starting any stream capture.  The
- *     plan's device must be the current device.
+ *     talks to the CUDA runtime; with lazy module loading it is also the moment the array becomes
+ *     resident on that device, so the driver's free-memory count drops by its size once); make
+ *     that first call before starting any stream capture.  Later calls neither allocate nor free.
+ *     The plan's device must be the current device.
  *   - All calls on a device share the one array.  Its contents are whatever the previous call
  *     left: the call clears the status words it needs at zero, and overwrites every pooled element
  *     its result depends on before reading it (metric tiles that reach past a sequence's last

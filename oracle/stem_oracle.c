@@ -25,6 +25,9 @@
  * of Eq. 2 and Eq. 4; pooled dot product equals the mean of the block's token
  * dot products; closed form of the magnitude term; beta = 0 ranking; brute-force
  * sort for selection; full budget reproduces dense causal softmax attention.
+ * Chunked prefill (so_*_chunk) is pinned against the one-shot functions: the rows of any split of a
+ * sequence into chunks must reproduce the one-shot lists bit for bit and the outputs to 1e-6; the
+ * group-shared metric (so_metric_shared) against a numpy fp64 mean of per-head metrics.
  * End-task accuracy (the paper's tables) needs trained weights: parity unpinned.
  *
  * Layouts
@@ -319,6 +322,217 @@ void so_attention(const uint16_t* Q, int64_t q_stride_tok, int64_t q_stride_head
             if (lse) lse[(int64_t)h * T + t0 + tq] = nk > 0 ? (float)(mx + log(denom)) : -INFINITY;
         }
         free(s); free(kpos); free(qd); free(acc);
+    }
+}
+
+/* =============================================================================================
+ * Chunked prefill with global token offsets (Conclusion, "Limitations and future work": the
+ * position-decay schedule is applied by keeping global token offsets across chunks).
+ *
+ * Sequence b is prefilled in chunks.  At one chunk, K and V hold the first kv_len(b) tokens of the
+ * sequence (packed by cu_kv), and Q holds only the chunk's tokens, positions q_start(b) ..
+ * kv_len(b)-1 (packed by cu_q; q_start is a multiple of the block size).  Block row r of the chunk
+ * is the GLOBAL row index r0(b) + local row, r0 = q_start / B; its causal blocks are 0 .. r of the
+ * prefix, and its budget is Eq. 3 evaluated at the global row of a sequence of N_total blocks (the
+ * caller passes k_eff already sliced to the chunk's rows).  Everything else is Algorithm 1 as above.
+ *
+ * Layouts: chunk rows are numbered sequence-major, RQ = rq_off(b) + (r - r0(b)); key blocks
+ * KB = kb_off(b) + j.  qbar [Hq, RQ_tot, d]; kbar [Hkv, KB_tot, d]; mv [Hkv, KB_tot].
+ * M [Hq, m_tot], m_tot = sum_b rows(b) * n_kv_blk(b); entry (h, b, r, j) at
+ *   h*m_tot + m_off(b) + (r - r0(b)) * n_kv_blk(b) + j, defined for j <= r.
+ * =========================================================================================== */
+void so_metric_chunk(const float* qbar, const float* kbar, const float* mv, int32_t Hq, int32_t Hkv, int32_t d,
+                     int32_t batch, const int32_t* n_kv_blk, const int32_t* r0, float beta, float score_scale,
+                     float* M) {
+    int64_t rq_tot = 0, kb_tot = 0, m_tot = 0;
+    for (int b = 0; b < batch; ++b) {
+        rq_tot += n_kv_blk[b] - r0[b];
+        kb_tot += n_kv_blk[b];
+        m_tot += (int64_t)(n_kv_blk[b] - r0[b]) * n_kv_blk[b];
+    }
+    int g = Hq / Hkv;
+    int64_t rq_off = 0, kb_off = 0, m_off = 0;
+    for (int b = 0; b < batch; ++b) {
+        int64_t nb = n_kv_blk[b], first = r0[b];
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+        for (int h = 0; h < Hq; ++h) {
+            for (int64_t r = first; r < nb; ++r) {
+                int kvh = h / g;
+                const float* qv = qbar + ((int64_t)h * rq_tot + rq_off + (r - first)) * d;
+                for (int64_t j = 0; j <= r; ++j) {
+                    const float* kv = kbar + ((int64_t)kvh * kb_tot + kb_off + j) * d;
+                    double acc = 0.0;
+                    for (int c = 0; c < d; ++c) acc += (double)qv[c] * (double)kv[c];
+                    double m = (double)score_scale * acc + (double)beta * (double)mv[(int64_t)kvh * kb_tot + kb_off + j];
+                    M[(int64_t)h * m_tot + m_off + (r - first) * nb + j] = (float)m;
+                }
+            }
+        }
+        rq_off += nb - first;
+        kb_off += nb;
+        m_off += (nb - first) * nb;
+    }
+}
+
+void so_select_chunk(const float* M, int32_t Hq, int32_t batch, const int32_t* n_kv_blk, const int32_t* r0,
+                     const int32_t* k_eff /*[RQ_tot]*/, int32_t stem, int32_t local, int32_t k_max,
+                     int32_t* sel_idx /*[Hq,RQ_tot,k_max]*/, int32_t* sel_cnt /*[Hq,RQ_tot]*/) {
+    int64_t rq_tot = 0, m_tot = 0;
+    for (int b = 0; b < batch; ++b) {
+        rq_tot += n_kv_blk[b] - r0[b];
+        m_tot += (int64_t)(n_kv_blk[b] - r0[b]) * n_kv_blk[b];
+    }
+    int64_t rq_off = 0, m_off = 0;
+    for (int b = 0; b < batch; ++b) {
+        int64_t nb = n_kv_blk[b], first = r0[b];
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+        for (int h = 0; h < Hq; ++h) {
+            for (int64_t r = first; r < nb; ++r) {
+                int64_t i = r + 1; /* the global row decides the forced blocks and the causal range */
+                int64_t n_stem = stem < i ? stem : i;
+                int64_t lo_local = i - local > 0 ? i - local : 0;
+                int64_t RQ = rq_off + (r - first);
+                int32_t ke = k_eff[RQ];
+                int32_t* out = sel_idx + ((int64_t)h * rq_tot + RQ) * k_max;
+                so_cand* cand = (so_cand*)malloc(sizeof(so_cand) * (size_t)i);
+                int n_out = 0, n_cand = 0;
+                for (int64_t j = 0; j < i; ++j) {
+                    if (j < n_stem || j >= lo_local) {
+                        out[n_out++] = (int32_t)j;
+                    } else {
+                        float m = M[(int64_t)h * m_tot + m_off + (r - first) * nb + j];
+                        if (m != m) m = -INFINITY;
+                        if (m == 0.0f) m = 0.0f;
+                        cand[n_cand].m = m;
+                        cand[n_cand].j = (int32_t)j;
+                        ++n_cand;
+                    }
+                }
+                int need = ke - n_out;
+                if (need > n_cand) need = n_cand;
+                if (need > 0) {
+                    qsort(cand, (size_t)n_cand, sizeof(so_cand), so_cand_cmp);
+                    for (int q = 0; q < need; ++q) out[n_out++] = cand[q].j;
+                }
+                free(cand);
+                qsort(out, (size_t)n_out, sizeof(int32_t), so_int_cmp);
+                for (int q = n_out; q < k_max; ++q) out[q] = -1;
+                sel_cnt[(int64_t)h * rq_tot + RQ] = n_out;
+            }
+        }
+        rq_off += nb - first;
+        m_off += (nb - first) * nb;
+    }
+}
+
+/* Attention of a chunk: the query token at chunk position tq has global position q_start + tq and
+ * sees the keys of its row's listed blocks with position <= its own.  O is [Tq, Hq, d] and lse
+ * [Hq, Tq], packed like Q.  rows: (h, RQ) pairs in the chunk's row numbering. */
+void so_attention_chunk(const uint16_t* Q, int64_t q_stride_tok, int64_t q_stride_head, const uint16_t* K,
+                        const uint16_t* V, int64_t kv_stride_tok, int64_t kv_stride_head, int32_t Hq, int32_t Hkv,
+                        int32_t d, int32_t batch, const int32_t* cu_q, const int32_t* cu_kv, const int32_t* q_start,
+                        int32_t B, const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_max,
+                        float softmax_scale, const int32_t* rows, int64_t n_rows, float* O, float* lse) {
+    int64_t rq_tot = 0, Tq = cu_q[batch];
+    for (int b = 0; b < batch; ++b) rq_tot += cdiv(cu_q[b + 1] - cu_q[b], B);
+    int g = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t it = 0; it < n_rows; ++it) {
+        int h = rows[2 * it], RQ = rows[2 * it + 1];
+        int kvh = h / g;
+        int b = 0;
+        int64_t rq_off = 0;
+        for (;; ++b) {
+            int64_t nr = cdiv(cu_q[b + 1] - cu_q[b], B);
+            if (RQ < rq_off + nr) break;
+            rq_off += nr;
+        }
+        int64_t tq0 = cu_q[b], nq = cu_q[b + 1] - cu_q[b];    /* chunk tokens of the sequence */
+        int64_t tk0 = cu_kv[b], nk_seq = cu_kv[b + 1] - cu_kv[b]; /* prefix tokens of the sequence */
+        int64_t start = q_start[b];
+        int64_t rl = RQ - rq_off;                                /* row inside the chunk */
+        const int32_t* list = sel_idx + ((int64_t)h * rq_tot + RQ) * k_max;
+        int cnt = sel_cnt[(int64_t)h * rq_tot + RQ];
+        int64_t max_keys = (int64_t)cnt * B;
+        double* s = (double*)malloc(sizeof(double) * (size_t)(max_keys > 0 ? max_keys : 1));
+        int64_t* kpos = (int64_t*)malloc(sizeof(int64_t) * (size_t)(max_keys > 0 ? max_keys : 1));
+        double* qd = (double*)malloc(sizeof(double) * (size_t)d);
+        double* acc = (double*)malloc(sizeof(double) * (size_t)d);
+        int64_t q_lo = rl * B, q_hi = q_lo + B < nq ? q_lo + B : nq;
+        for (int64_t tq = q_lo; tq < q_hi; ++tq) {
+            int64_t pos = start + tq; /* global position of the query token */
+            const uint16_t* qp = Q + (tq0 + tq) * q_stride_tok + (int64_t)h * q_stride_head;
+            for (int c = 0; c < d; ++c) qd[c] = (double)bf16_to_f32(qp[c]);
+            int64_t nk = 0;
+            double mx = -INFINITY;
+            for (int e = 0; e < cnt; ++e) {
+                int64_t j = list[e];
+                int64_t k_lo = j * B, k_hi = k_lo + B < nk_seq ? k_lo + B : nk_seq;
+                for (int64_t tk = k_lo; tk < k_hi && tk <= pos; ++tk) {
+                    const uint16_t* kp = K + (tk0 + tk) * kv_stride_tok + (int64_t)kvh * kv_stride_head;
+                    double dot = 0.0;
+#pragma omp simd reduction(+ : dot)
+                    for (int c = 0; c < d; ++c) dot += qd[c] * (double)bf16_to_f32(kp[c]);
+                    double sc = dot * (double)softmax_scale;
+                    s[nk] = sc;
+                    kpos[nk] = tk;
+                    ++nk;
+                    if (sc > mx) mx = sc;
+                }
+            }
+            for (int c = 0; c < d; ++c) acc[c] = 0.0;
+            double denom = 0.0;
+            for (int64_t e = 0; e < nk; ++e) {
+                double p = exp(s[e] - mx);
+                denom += p;
+                const uint16_t* vp = V + (tk0 + kpos[e]) * kv_stride_tok + (int64_t)kvh * kv_stride_head;
+#pragma omp simd
+                for (int c = 0; c < d; ++c) acc[c] += p * (double)bf16_to_f32(vp[c]);
+            }
+            float* op = O + ((tq0 + tq) * (int64_t)Hq + h) * d;
+            for (int c = 0; c < d; ++c) op[c] = nk > 0 ? (float)(acc[c] / denom) : 0.0f;
+            if (lse) lse[(int64_t)h * Tq + tq0 + tq] = nk > 0 ? (float)(mx + log(denom)) : -INFINITY;
+        }
+        free(s); free(kpos); free(qd); free(acc);
+    }
+}
+
+/* =============================================================================================
+ * Group-shared selection (Main Results: the integration into a model whose block-level top-k is
+ * shared by the query heads of a GQA group).  One index list per (kv head, row) instead of one per
+ * query head.  The paper does not say how the heads' metrics are combined; the reading taken here:
+ * the group's metric is the MEAN over its query heads of Eq. 7's metric,
+ *   Mg[kvh, r, j] = (1/g) * sum_{h in group} ( score_scale * Qbar[h,r].Kbar[kvh,j] ) + beta * MV[kvh,j],
+ * which equals Eq. 7 evaluated on the group-mean pooled query.  Layout of Mg: that of M with Hkv heads.
+ * =========================================================================================== */
+void so_metric_shared(const float* qbar /*[Hq,R_tot,d]*/, const float* kbar /*[Hkv,R_tot,d]*/,
+                      const float* mv /*[Hkv,R_tot]*/, int32_t Hq, int32_t Hkv, int32_t d, int32_t batch,
+                      const int32_t* n_blk, float beta, float score_scale, float* Mg /*[Hkv,m_tot]*/) {
+    int64_t r_tot = 0, m_tot = 0;
+    for (int b = 0; b < batch; ++b) { r_tot += n_blk[b]; m_tot += (int64_t)n_blk[b] * n_blk[b]; }
+    int g = Hq / Hkv;
+    int64_t row_off = 0, m_off = 0;
+    for (int b = 0; b < batch; ++b) {
+        int64_t nb = n_blk[b];
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+        for (int kvh = 0; kvh < Hkv; ++kvh) {
+            for (int64_t r = 0; r < nb; ++r) {
+                for (int64_t j = 0; j <= r; ++j) {
+                    const float* kv = kbar + ((int64_t)kvh * r_tot + row_off + j) * d;
+                    double sum = 0.0;
+                    for (int q = 0; q < g; ++q) {
+                        const float* qv = qbar + ((int64_t)(kvh * g + q) * r_tot + row_off + r) * d;
+                        double acc = 0.0;
+                        for (int c = 0; c < d; ++c) acc += (double)qv[c] * (double)kv[c];
+                        sum += acc;
+                    }
+                    double m = (double)score_scale * (sum / (double)g) + (double)beta * (double)mv[(int64_t)kvh * r_tot + row_off + j];
+                    Mg[(int64_t)kvh * m_tot + m_off + r * nb + j] = (float)m;
+                }
+            }
+        }
+        row_off += nb;
+        m_off += nb * nb;
     }
 }
 

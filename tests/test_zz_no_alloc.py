@@ -20,6 +20,7 @@ pytestmark = pytest.mark.gpu
 
 def _metric_triple(w):
     """M of the workload from stem_score (caller workspace), stem_score_static and the checker."""
+    _first_call_set_up()
     data = wl.make_qkv(w)
     plan = StemPlan.from_workload(w)
     q, k, v = to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"])
@@ -39,6 +40,25 @@ def _metric_triple(w):
     assert binding.stem_check_status(plan, static_scratch=True)[0] == binding.STEM_OK
     ref, *_ = so.score(data["q"], data["k"], data["v"], data["cu_seqlens"], oracle_params(w))
     return want.cpu().numpy(), got.cpu().numpy(), ref
+
+
+_set_up_done = False
+
+
+def _first_call_set_up():
+    """The documented one-time set-up: the first call on a device resolves the address of the built-in array
+    (with CUDA's lazy module loading that is also the moment the array itself becomes resident).  It is made
+    here on a tiny problem so that the calls under test are ordinary, later calls."""
+    global _set_up_done
+    if _set_up_done:
+        return
+    w = wl.small("noalloc_setup", seqlens=(300,), hq=2, hkv=1, block=64, permille=500)
+    data = wl.make_qkv(w)
+    plan = StemPlan.from_workload(w)
+    m = torch.empty((w.num_q_heads, plan.info.metric_elems), dtype=torch.float32, device="cuda")
+    binding.stem_score_static(plan, to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"]), m)
+    torch.cuda.synchronize()
+    _set_up_done = True
 
 
 def _assert_close(want, got):
