@@ -10,6 +10,10 @@
  *   stem_sparse_prefill  Alg. 1 step 3d: exact causal softmax attention over the listed blocks
  *   stem_score_select    steps 1-3c in one call
  *   stem_prefill         all of Algorithm 1, ordered on one stream, no host synchronisation
+ *   stem_plan_create_ex  the same path for a CHUNK of every sequence against its K / V prefix, with the
+ *                        budget taken at the global token offset (the paper's Conclusion), with the pooled
+ *                        K-side tensors in a caller-owned cache (stem_pool_kv, *_cached), and with one
+ *                        index list per GQA group (the block-level top-k shared per group of Main Results)
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned.
@@ -21,8 +25,8 @@
  *   - Query-block rows are numbered globally, sequence-major: R = row_offset(b) + r,
  *     r = 0 .. N_blk(b)-1, N_blk(b) = ceil(len_b / block); R_tot = sum_b N_blk(b).
  *   - Index lists: sel_idx is int32 [num_q_heads, R_tot, k_max], sel_cnt int32
- *     [num_q_heads, R_tot].  Row (h, R) holds sel_cnt valid block ids, local to the
- *     sequence, strictly ascending, each <= r; the remaining entries are -1.
+ *     [num_q_heads, R_tot] (num_kv_heads instead with share_group).  Row (h, R) holds sel_cnt valid
+ *     block ids, local to the sequence, strictly ascending, each <= r; the remaining entries are -1.
  *   - `stream` is a cudaStream_t passed as void*.  Hot calls enqueue work on it and return;
  *     they never allocate, never synchronise and never throw.
  *   - Return value: STEM_OK (0) or a negative stem_status.  Nothing is enqueued when a call
@@ -83,21 +87,57 @@ typedef struct stem_plan stem_plan; /* opaque; owns small host and device tables
 /* Sizes a caller needs to allocate buffers for a plan. */
 typedef struct {
   size_t workspace_bytes;       /* scratch the hot calls need (pooled tensors, metric, lists, status) */
-  int32_t total_tokens;         /* T                                                               */
-  int32_t total_q_blocks;       /* R_tot                                                           */
+  int32_t total_tokens;         /* tokens of Q and O (the chunk's tokens with chunked prefill)      */
+  int32_t total_q_blocks;       /* R_tot: query-block rows                                         */
   int32_t k_max;                /* longest index list = max_r k_eff(r)                             */
-  int64_t metric_elems;         /* per head: sum_b N_blk(b)^2, the size of one head of M           */
-  int64_t selected_blocks;      /* sum over heads and rows of the list lengths (exact)             */
-  int64_t causal_blocks;        /* sum over heads and rows of r+1 (admissible blocks)              */
+  int64_t metric_elems;         /* per head: sum_b rows(b) * N_blk(b), the size of one head of M   */
+  int64_t selected_blocks;      /* sum over query heads and rows of the list lengths (exact)       */
+  int64_t causal_blocks;        /* sum over query heads and rows of r+1 (admissible blocks)        */
   int64_t selected_pairs;       /* unmasked (query, key) pairs inside the selected blocks          */
   int64_t causal_pairs;         /* unmasked (query, key) pairs of dense causal attention           */
+  int32_t total_kv_tokens;      /* tokens of K and V (= total_tokens without chunks)               */
+  int32_t list_heads;           /* first dimension of sel_idx / sel_cnt / M: H_q, or H_kv with share_group */
+  size_t kcache_bytes;          /* size of the caller-owned pooled-K cache (0 without one)         */
+  int32_t total_key_blocks;     /* key blocks of all sequences (sum_b N_blk(b))                    */
+  int32_t new_key_blocks;       /* key blocks the chunk adds (what stem_pool_kv pools)             */
 } stem_plan_info;
+
+/* Extensions of the problem statement (all optional; a zeroed struct or NULL means plain Algorithm 1).
+ *
+ * Chunked prefill (Conclusion, "Limitations and future work": the position-decay schedule applies to chunk
+ * prefill when global token offsets are kept across chunks).  cfg.cu_seqlens_host then describes K and V: the
+ * first kv_len(b) tokens of every sequence.  Q and O hold only the chunk, the tokens q_start(b) ..
+ * kv_len(b)-1 of every sequence, packed in sequence order.  Block row r of a chunk is the global row
+ * (r >= q_start/B): its causal blocks are 0 .. r of the prefix, and its budget is Eq. 3 at row r+1 of a
+ * sequence of ceil(total_len(b)/B) blocks, with k_start taken from that block count.
+ *
+ * Pooled-K cache (Main Results / Related Work: block-level K-side representations kept with the KV cache).
+ * With kcache_blocks_per_seq > 0 the K-side tensors of step 1 (Kbar parts and MV) live in caller memory of
+ * stem_plan_info.kcache_bytes: sequence b owns rows b*capacity .. of it, row j = its block j, so the layout
+ * does not move while the prefix grows.  stem_pool_kv writes the rows of the blocks the plan's chunk adds;
+ * the *_cached calls read rows 0 .. N_blk(b)-1 and never touch K or V for scoring.
+ *
+ * share_group (Main Results: integration with a block-level top-k shared by the heads of a GQA group): one
+ * index list per (kv head, row).  The group's metric is the mean over its query heads of Eq. 7, i.e. Eq. 7 on
+ * the group-mean pooled query; sel_idx / sel_cnt / M have num_kv_heads heads; every query head of the group
+ * attends over its group's list. */
+typedef struct {
+  const int32_t* q_start_host;    /* HOST [batch]: first query token of every sequence's chunk, a multiple of
+                                     block, < kv_len(b); NULL = 0 (no chunking)                               */
+  const int32_t* total_len_host;  /* HOST [batch]: full length of every sequence for Eq. 3, >= kv_len(b);
+                                     NULL = kv_len(b)                                                         */
+  int32_t kcache_blocks_per_seq;  /* capacity (blocks per sequence) of a caller-owned pooled-K cache; 0 = none */
+  int32_t share_group;            /* 1: one index list per kv head                                            */
+  int32_t reserved[4];            /* must be 0                                                                */
+} stem_options;
 
 /* Builds the per-row budget table k_eff(r) (Eq. 3 in block units, i = r+1, clamped by the forced
  * blocks, min_blocks and the r+1 causal blocks), the row maps and the work order of the attention
  * kernel, and uploads them to the current CUDA device (the only allocation the library makes).
  * Host work only plus one synchronous copy; call it outside the hot path. */
 int stem_plan_create(const stem_config* cfg, stem_plan** out_plan);
+/* The same with the extensions above; opts == NULL is stem_plan_create. */
+int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_plan** out_plan);
 int stem_plan_destroy(stem_plan* plan);
 int stem_plan_query(const stem_plan* plan, stem_plan_info* info);
 
@@ -186,6 +226,24 @@ int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, con
  * synchronisation.  sel_idx / sel_cnt are optional outputs (both NULL: lists stay in the workspace). */
 int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
                  int32_t* sel_cnt, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+/* K side of Alg. 1 step 1 into a caller-owned pooled-K cache (plans created with kcache_blocks_per_seq > 0):
+ * block means of K (as the three bf16 parts the metric kernel multiplies) and MV = max(0, max ln ||V||) for
+ * the key blocks the plan's chunk adds (every block without chunking), read from the packed K / V of the
+ * prefix.  The hook for "pool K and V once, when they are written".  kcache: DEVICE, 256-byte aligned,
+ * stem_plan_info.kcache_bytes; rows of other blocks are left as they are. */
+int stem_pool_kv(const stem_plan* plan, const void* K, const void* V, void* kcache, void* stream);
+
+/* Alg. 1 steps 1-3c reading only Q: pools Q, takes Kbar and MV of blocks 0 .. N_blk(b)-1 from the cache
+ * (written by earlier stem_pool_kv calls), metric, budget, selection.  Same lists as stem_score_select. */
+int stem_score_select_cached(const stem_plan* plan, const void* Q, const void* kcache, int32_t* sel_idx,
+                             int32_t* sel_cnt, void* workspace, size_t workspace_bytes, void* stream);
+
+/* All of Algorithm 1 with the cache: update_cache != 0 first pools the chunk's new key blocks into it
+ * (stem_pool_kv), then stem_score_select_cached and stem_sparse_prefill, ordered on `stream`. */
+int stem_prefill_cached(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, void* kcache,
+                        int update_cache, int32_t* sel_idx, int32_t* sel_cnt, float* lse, void* workspace,
+                        size_t workspace_bytes, void* stream);
 
 /* Synchronises `stream`, then reads the device status words of `workspace` (workspace == NULL: of
  * the scratch built into the library, see stem_score_static) and clears them if they are set.

@@ -6,6 +6,7 @@ seeded synthetic workloads used by the tests and the benchmark.
 """
 from . import workloads  # noqa: F401
 from .binding import (  # noqa: F401
-    StemConfig, StemError, StemPlan, StemPlanInfo, load, library_path, status_string,
-    stem_check_status, stem_prefill, stem_score, stem_score_static, stem_select, stem_score_select, stem_sparse_prefill,
+    StemConfig, StemError, StemOptions, StemPlan, StemPlanInfo, load, library_path, status_string,
+    stem_check_status, stem_pool_kv, stem_prefill, stem_prefill_cached, stem_score, stem_score_select,
+    stem_score_select_cached, stem_score_static, stem_select, stem_sparse_prefill,
 )

@@ -23,7 +23,8 @@ STEM_ERR_DEVICE_TIMEOUT = -5
 STEM_ERR_STATIC_SCRATCH = -6
 STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
-EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_destroy", "stem_plan_query",
+EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_create_ex", "stem_plan_destroy", "stem_plan_query",
+           "stem_pool_kv", "stem_score_select_cached", "stem_prefill_cached",
            "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_score_select", "stem_sparse_prefill", "stem_prefill",
            "stem_check_status", "stem_selftest_wait_timeout", "stem_last_launch_count")
 
@@ -64,6 +65,21 @@ class StemPlanInfo(ctypes.Structure):
         ("causal_blocks", ctypes.c_int64),
         ("selected_pairs", ctypes.c_int64),
         ("causal_pairs", ctypes.c_int64),
+        ("total_kv_tokens", ctypes.c_int32),
+        ("list_heads", ctypes.c_int32),
+        ("kcache_bytes", ctypes.c_size_t),
+        ("total_key_blocks", ctypes.c_int32),
+        ("new_key_blocks", ctypes.c_int32),
+    ]
+
+
+class StemOptions(ctypes.Structure):
+    _fields_ = [
+        ("q_start_host", ctypes.POINTER(ctypes.c_int32)),
+        ("total_len_host", ctypes.POINTER(ctypes.c_int32)),
+        ("kcache_blocks_per_seq", ctypes.c_int32),
+        ("share_group", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 4),
     ]
 
 
@@ -95,6 +111,10 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_status_string.restype = ctypes.c_char_p
     lib.stem_status_string.argtypes = [ctypes.c_int]
     lib.stem_plan_create.argtypes = [ctypes.POINTER(StemConfig), ctypes.POINTER(vp)]
+    lib.stem_plan_create_ex.argtypes = [ctypes.POINTER(StemConfig), ctypes.POINTER(StemOptions), ctypes.POINTER(vp)]
+    lib.stem_pool_kv.argtypes = [vp, vp, vp, vp, vp]
+    lib.stem_score_select_cached.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.stem_prefill_cached.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_plan_destroy.argtypes = [vp]
     lib.stem_plan_query.argtypes = [vp, ctypes.POINTER(StemPlanInfo)]
     lib.stem_plan_budget.argtypes = [vp, i32p]
@@ -138,7 +158,13 @@ class StemPlan:
     def __init__(self, seqlens: Sequence[int], num_q_heads: int, num_kv_heads: int, block: int = 128,
                  budget_permille: int = 100, k_start_blocks: int = 0, mu=(7, 10), stem_blocks: int = 4,
                  local_blocks: int = 4, min_blocks: int = 0, beta: float = 0.2, score_scale: float = 0.0,
-                 softmax_scale: float = 0.0, head_dim: int = 128, q_strides=None, kv_strides=None):
+                 softmax_scale: float = 0.0, head_dim: int = 128, q_strides=None, kv_strides=None,
+                 q_starts: Optional[Sequence[int]] = None, total_lens: Optional[Sequence[int]] = None,
+                 kcache_blocks_per_seq: int = 0, share_group: bool = False):
+        """``seqlens`` are the lengths of K and V.  With ``q_starts`` (chunked prefill) Q and O hold only the
+        tokens q_start(b) .. seqlens[b]-1 of every sequence and ``total_lens`` are the full sequence lengths the
+        budget schedule is evaluated on; ``kcache_blocks_per_seq`` > 0 puts the pooled K-side tensors into a
+        caller-owned cache (``stem_pool_kv`` / ``*_cached``); ``share_group`` selects one list per kv head."""
         lib = load()
         cu = [0]
         for n in seqlens:
@@ -158,7 +184,16 @@ class StemPlan:
         cfg.kv_stride_tok, cfg.kv_stride_head = ks
         self.config = cfg
         self._h = ctypes.c_void_p()
-        _check(lib.stem_plan_create(ctypes.byref(cfg), ctypes.byref(self._h)), "stem_plan_create")
+        opts = StemOptions()
+        if q_starts is not None:
+            self._qs = (ctypes.c_int32 * len(seqlens))(*[int(x) for x in q_starts])
+            opts.q_start_host = ctypes.cast(self._qs, ctypes.POINTER(ctypes.c_int32))
+        if total_lens is not None:
+            self._tl = (ctypes.c_int32 * len(seqlens))(*[int(x) for x in total_lens])
+            opts.total_len_host = ctypes.cast(self._tl, ctypes.POINTER(ctypes.c_int32))
+        opts.kcache_blocks_per_seq = int(kcache_blocks_per_seq)
+        opts.share_group = 1 if share_group else 0
+        _check(lib.stem_plan_create_ex(ctypes.byref(cfg), ctypes.byref(opts), ctypes.byref(self._h)), "stem_plan_create_ex")
         info = StemPlanInfo()
         _check(lib.stem_plan_query(self._h, ctypes.byref(info)), "stem_plan_query")
         self.info = info
@@ -237,6 +272,28 @@ def stem_score_select(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch
     p, n = _ws_args(plan, workspace)
     _check(load().stem_score_select(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(sel_idx), _ptr(sel_cnt), p, n,
                                     _stream()), "stem_score_select")
+
+
+def stem_pool_kv(plan: StemPlan, k: torch.Tensor, v: torch.Tensor, kcache: torch.Tensor) -> None:
+    """K side of step 1 for the key blocks the plan's chunk adds, into the caller-owned pooled-K cache."""
+    _check(load().stem_pool_kv(plan.handle, _ptr(k), _ptr(v), _ptr(kcache), _stream()), "stem_pool_kv")
+
+
+def stem_score_select_cached(plan: StemPlan, q: torch.Tensor, kcache: torch.Tensor, sel_idx: torch.Tensor,
+                             sel_cnt: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> None:
+    p, n = _ws_args(plan, workspace)
+    _check(load().stem_score_select_cached(plan.handle, _ptr(q), _ptr(kcache), _ptr(sel_idx), _ptr(sel_cnt), p, n,
+                                           _stream()), "stem_score_select_cached")
+
+
+def stem_prefill_cached(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor,
+                        kcache: torch.Tensor, update_cache: bool = True, sel_idx: Optional[torch.Tensor] = None,
+                        sel_cnt: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None) -> None:
+    p, n = _ws_args(plan, workspace)
+    _check(load().stem_prefill_cached(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kcache),
+                                      1 if update_cache else 0, _ptr(sel_idx), _ptr(sel_cnt), _ptr(lse), p, n, _stream()),
+           "stem_prefill_cached")
 
 
 def stem_sparse_prefill(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

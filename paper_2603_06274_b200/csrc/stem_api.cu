@@ -92,11 +92,26 @@ const char* stem_status_string(int s) {
   }
 }
 
-int stem_plan_create(const stem_config* cfg, stem_plan** out) {
+int stem_plan_create(const stem_config* cfg, stem_plan** out) { return stem_plan_create_ex(cfg, nullptr, out); }
+
+int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_plan** out) {
   if (!out) return STEM_ERR_INVALID_ARG;
   *out = nullptr;
   int rc = validate(cfg);
   if (rc != STEM_OK) return rc;
+  stem_options o{};
+  if (opts) o = *opts;
+  for (int i = 0; i < 4; ++i)
+    if (o.reserved[i] != 0) return STEM_ERR_INVALID_ARG;
+  if (o.kcache_blocks_per_seq < 0 || (o.share_group != 0 && o.share_group != 1)) return STEM_ERR_INVALID_ARG;
+  const int B = cfg->block, batch = cfg->batch, Hq = cfg->num_q_heads, Hkv = cfg->num_kv_heads;
+  for (int b = 0; b < batch; ++b) {
+    const int64_t kv_len = cfg->cu_seqlens_host[b + 1] - cfg->cu_seqlens_host[b];
+    const int64_t q0 = o.q_start_host ? o.q_start_host[b] : 0;
+    const int64_t tot = o.total_len_host ? o.total_len_host[b] : kv_len;
+    if (q0 < 0 || q0 >= kv_len || q0 % B != 0 || tot < kv_len) return STEM_ERR_INVALID_ARG;
+    if (o.kcache_blocks_per_seq > 0 && (kv_len + B - 1) / B > o.kcache_blocks_per_seq) return STEM_ERR_INVALID_ARG;
+  }
 
   stem_plan* sp = new (std::nothrow) stem_plan();
   if (!sp) return STEM_ERR_CUDA;
@@ -106,35 +121,49 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.cfg.cu_seqlens_host = nullptr;
   p.score_scale = cfg->score_scale == 0.f ? 1.f : cfg->score_scale;
   p.softmax_scale = cfg->softmax_scale == 0.f ? 1.f / std::sqrt((float)kHeadDim) : cfg->softmax_scale;
+  p.kcache_blocks = o.kcache_blocks_per_seq;
+  p.share_group = o.share_group != 0;
+  p.H_list = p.share_group ? Hkv : Hq;
 
-  const int B = cfg->block, batch = cfg->batch, Hq = cfg->num_q_heads, Hkv = cfg->num_kv_heads;
   const int g = Hq / Hkv;
-  p.T = p.cu[batch];
+  p.T_kv = p.cu[batch];
 
-  std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_len(batch), seq_nblk(batch),
-      seq_row_off(batch);
+  std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_nblk(batch), seq_r0(batch),
+      seq_row_off(batch), seq_kb_off(batch), kb_tok0, kb_ntok, kb_dst, kb_new;
   std::vector<int64_t> seq_m_off(batch), seq_mt_off(batch);
   int64_t m_off = 0, mt_off = 0;
+  int32_t q_tok = 0, kb_off = 0;
   for (int b = 0; b < batch; ++b) {
-    const int32_t n = p.cu[b + 1] - p.cu[b];
-    const int32_t nb = (n + B - 1) / B;
+    const int32_t n = p.cu[b + 1] - p.cu[b];           // tokens of the K / V prefix
+    const int32_t nb = (n + B - 1) / B;                // its blocks
+    const int32_t q0 = o.q_start_host ? o.q_start_host[b] : 0;
+    const int32_t r0 = q0 / B;
+    const int64_t n_tot = o.total_len_host ? o.total_len_host[b] : n;
+    const int64_t nb_tot = (n_tot + B - 1) / B;        // blocks of the whole sequence: N of Eq. 3
     seq_tok0[b] = p.cu[b];
-    seq_len[b] = n;
     seq_nblk[b] = nb;
+    seq_r0[b] = r0;
     seq_row_off[b] = (int32_t)row_seq.size();
+    seq_kb_off[b] = p.kcache_blocks > 0 ? b * p.kcache_blocks : kb_off;
     seq_m_off[b] = m_off;
     seq_mt_off[b] = mt_off;
-    mt_off += (int64_t)nb * ((nb + 31) / 32 * 32);  // rows padded to whole 32-column groups
-    m_off += (int64_t)nb * nb;
+    mt_off += (int64_t)(nb - r0) * ((nb + 31) / 32 * 32);  // rows padded to whole 32-column groups
+    m_off += (int64_t)(nb - r0) * nb;
     p.max_nblk = std::max(p.max_nblk, nb);
-    const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb) / 1000;
-    for (int32_t r = 0; r < nb; ++r) {
+    const int64_t k_s = cfg->k_start_blocks > 0 ? cfg->k_start_blocks : ((int64_t)cfg->budget_permille * nb_tot) / 1000;
+    for (int32_t j = 0; j < nb; ++j) {
+      if (j >= r0) kb_new.push_back((int32_t)kb_tok0.size());
+      kb_tok0.push_back(p.cu[b] + j * B);
+      kb_ntok.push_back(std::min(B, n - j * B));
+      kb_dst.push_back(seq_kb_off[b] + j);
+    }
+    for (int32_t r = r0; r < nb; ++r) {
       row_seq.push_back(b);
       row_r.push_back(r);
-      row_tok0.push_back(p.cu[b] + r * B);
+      row_tok0.push_back(q_tok + (r - r0) * B);
       const int32_t ntok = std::min(B, n - r * B);
       row_ntok.push_back(ntok);
-      const int32_t ke = budget_row(r + 1, nb, k_s, *cfg);
+      const int32_t ke = budget_row(r + 1, nb_tot, k_s, *cfg);
       p.k_eff.push_back(ke);
       p.k_max = std::max(p.k_max, ke);
       const int64_t diag = (int64_t)ntok * (ntok + 1) / 2;
@@ -143,8 +172,14 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
       p.selected_pairs += (int64_t)(ke - 1) * ntok * B + diag;
       p.causal_pairs += (int64_t)r * ntok * B + diag;
     }
+    q_tok += n - q0;
+    kb_off += nb;
   }
+  p.T = q_tok;
   p.R_tot = (int32_t)row_seq.size();
+  p.n_kb_all = (int32_t)kb_tok0.size();
+  p.n_kb_new = (int32_t)kb_new.size();
+  p.KB_tot = p.kcache_blocks > 0 ? batch * p.kcache_blocks : kb_off;
   p.m_tot = m_off;
   p.mt_tot = mt_off;
   p.selected_blocks *= Hq;
@@ -157,15 +192,19 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     return STEM_ERR_UNSUPPORTED;
   }
 
-  // Tiles of the metric GEMM: the 128 x 128 tiles of every sequence's causal triangle, long rows first.
+  // Tiles of the metric GEMM: 128 query rows x 128 key blocks, the tiles of every sequence that hold a causal
+  // entry (j <= r for some row of the tile), long rows first.
   std::vector<int32_t> gemm_tiles;
   {
     int max_t = 0;
-    for (int b = 0; b < batch; ++b) max_t = std::max(max_t, (seq_nblk[b] + 127) / 128);
+    for (int b = 0; b < batch; ++b) max_t = std::max(max_t, (seq_nblk[b] - seq_r0[b] + 127) / 128);
     for (int ti = max_t - 1; ti >= 0; --ti)
-      for (int b = 0; b < batch; ++b)
-        if (ti < (seq_nblk[b] + 127) / 128)
-          for (int tj = 0; tj <= ti; ++tj) { gemm_tiles.push_back(b); gemm_tiles.push_back(ti); gemm_tiles.push_back(tj); }
+      for (int b = 0; b < batch; ++b) {
+        const int rows_b = seq_nblk[b] - seq_r0[b];
+        if (ti >= (rows_b + 127) / 128) continue;
+        const int r_last = seq_r0[b] + std::min(rows_b, (ti + 1) * 128) - 1;  // largest global row of the tile
+        for (int tj = 0; tj <= r_last / 128; ++tj) { gemm_tiles.push_back(b); gemm_tiles.push_back(ti); gemm_tiles.push_back(tj); }
+      }
     p.n_gemm_tiles = (int32_t)(gemm_tiles.size() / 3);
   }
 
@@ -187,16 +226,17 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
     p.n_items = p.R_tot * Hq;
   }
 
-  // Workspace layout.
+  // Workspace layout.  With a caller-owned cache the K-side tensors are not part of the workspace.
   {
+    const bool own_k = p.kcache_blocks == 0;
     size_t off = 0;
     p.ws.status = off; off = align_up(off + kStatusWords * 4, 256);
-    p.ws.mv = off;     off = align_up(off + (size_t)Hkv * p.R_tot * 4, 256);
-    p.ws.qsplit = off; off = align_up(off + (size_t)3 * Hq * p.R_tot * kHeadDim * 2, 256);
-    p.ws.ksplit = off; off = align_up(off + (size_t)3 * Hkv * p.R_tot * kHeadDim * 2, 256);
-    p.ws.metric = off; off = align_up(off + (size_t)Hq * (size_t)p.mt_tot * 4, 256);
-    p.ws.sel_idx = off; off = align_up(off + (size_t)Hq * p.R_tot * p.k_max * 4, 256);
-    p.ws.sel_cnt = off; off = align_up(off + (size_t)Hq * p.R_tot * 4, 256);
+    p.ws.mv = off;     off = align_up(off + (own_k ? (size_t)Hkv * p.KB_tot * 4 : 0), 256);
+    p.ws.qsplit = off; off = align_up(off + (size_t)3 * p.H_list * p.R_tot * kHeadDim * 2, 256);
+    p.ws.ksplit = off; off = align_up(off + (own_k ? (size_t)3 * Hkv * p.KB_tot * kHeadDim * 2 : 0), 256);
+    p.ws.metric = off; off = align_up(off + (size_t)p.H_list * (size_t)p.mt_tot * 4, 256);
+    p.ws.sel_idx = off; off = align_up(off + (size_t)p.H_list * p.R_tot * p.k_max * 4, 256);
+    p.ws.sel_cnt = off; off = align_up(off + (size_t)p.H_list * p.R_tot * 4, 256);
     p.ws.total = off;
   }
 
@@ -210,10 +250,11 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   std::vector<uint8_t> blob;
   const size_t o_row_seq = push(blob, row_seq), o_row_r = push(blob, row_r), o_row_tok0 = push(blob, row_tok0),
                o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
-               o_seq_len = push(blob, seq_len), o_seq_nblk = push(blob, seq_nblk),
-               o_seq_row_off = push(blob, seq_row_off), o_seq_m_off = push(blob, seq_m_off), o_seq_mt_off = push(blob, seq_mt_off),
-               o_gt = push(blob, gemm_tiles), o_ws = push(blob, work_sparse),
-               o_wd = push(blob, work_dense);
+               o_seq_nblk = push(blob, seq_nblk), o_seq_r0 = push(blob, seq_r0), o_seq_row_off = push(blob, seq_row_off),
+               o_seq_kb_off = push(blob, seq_kb_off), o_seq_m_off = push(blob, seq_m_off),
+               o_seq_mt_off = push(blob, seq_mt_off), o_kb_tok0 = push(blob, kb_tok0), o_kb_ntok = push(blob, kb_ntok),
+               o_kb_dst = push(blob, kb_dst), o_kb_new = push(blob, kb_new), o_gt = push(blob, gemm_tiles),
+               o_ws = push(blob, work_sparse), o_wd = push(blob, work_dense);
   if (cudaMalloc(&p.d_blob, blob.size()) != cudaSuccess ||
       cudaMemcpy(p.d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
     cudaGetLastError();
@@ -228,11 +269,16 @@ int stem_plan_create(const stem_config* cfg, stem_plan** out) {
   p.rows.row_ntok = (const int32_t*)(d + o_row_ntok);
   p.rows.row_keff = (const int32_t*)(d + o_keff);
   p.rows.seq_tok0 = (const int32_t*)(d + o_seq_tok0);
-  p.rows.seq_len = (const int32_t*)(d + o_seq_len);
   p.rows.seq_nblk = (const int32_t*)(d + o_seq_nblk);
+  p.rows.seq_r0 = (const int32_t*)(d + o_seq_r0);
   p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
+  p.rows.seq_kb_off = (const int32_t*)(d + o_seq_kb_off);
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
   p.rows.seq_mt_off = (const int64_t*)(d + o_seq_mt_off);
+  p.rows.kb_tok0 = (const int32_t*)(d + o_kb_tok0);
+  p.rows.kb_ntok = (const int32_t*)(d + o_kb_ntok);
+  p.rows.kb_dst = (const int32_t*)(d + o_kb_dst);
+  p.rows.kb_new = (const int32_t*)(d + o_kb_new);
   p.d_gemm_tiles = (const int32_t*)(d + o_gt);
   p.d_work_sparse = (const int32_t*)(d + o_ws);
   p.d_work_dense = (const int32_t*)(d + o_wd);
@@ -258,6 +304,11 @@ int stem_plan_query(const stem_plan* plan, stem_plan_info* info) {
   info->causal_blocks = p.causal_blocks;
   info->selected_pairs = p.selected_pairs;
   info->causal_pairs = p.causal_pairs;
+  info->total_kv_tokens = p.T_kv;
+  info->list_heads = p.H_list;
+  info->kcache_bytes = p.kcache_blocks > 0 ? kcache_bytes(p) : 0;
+  info->total_key_blocks = p.n_kb_all;
+  info->new_key_blocks = p.n_kb_new;
   return STEM_OK;
 }
 
@@ -297,22 +348,32 @@ static int check_ws(const Plan& p, const void* ws, size_t bytes) {
 
 static int cuda_rc(cudaError_t e) { return e == cudaSuccess ? STEM_OK : STEM_ERR_CUDA; }
 
-// Alg. 1 steps 1-3c on one stream: pooling (one pass over Q, K, V; also emits the pooled vectors as
-// bf16 parts), the metric of every causal block on the tensor cores into the workspace (stored as
-// bit planes of the selection's order-preserving keys), and the row-wise selection from it.
-// (Two ways of overlapping the HBM-bound pooling with the scoring were measured and dropped: phases
+// Where the K-side tensors of step 1 live: in the workspace, or in the caller's pooled-K cache.
+struct KSide {
+  void* ksplit;
+  float* mv;
+};
+static KSide k_side(const Plan& p, uint8_t* w, void* kcache) {
+  if (kcache) return {kcache, (float*)((uint8_t*)kcache + kcache_mv_offset(p))};
+  return {w + p.ws.ksplit, (float*)(w + p.ws.mv)};
+}
+
+// Alg. 1 steps 1-3c on one stream: pooling (one pass over Q and, unless the K side comes from a cache, over K
+// and V; emits the pooled vectors as bf16 parts), the metric of every causal block on the tensor cores into
+// the workspace (stored as bit planes of the selection's order-preserving keys), and the row-wise selection
+// from it.  (Two ways of overlapping the HBM-bound pooling with the scoring were measured and dropped: phases
 // on two streams lose more to cross-stream event waits than they gain, and one persistent kernel
 // with a shared ticket list leaves too few warps per SM to stream HBM.)
-static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, uint8_t* w, int32_t* idx,
-                                int32_t* cnt, cudaStream_t s) {
-  float* mv = (float*)(w + p.ws.mv);
+static int enqueue_score_select(const Plan& p, const void* Q, const void* K, const void* V, void* kcache, uint8_t* w,
+                                int32_t* idx, int32_t* cnt, cudaStream_t s) {
+  const KSide ks = k_side(p, w, kcache);
   float* M = (float*)(w + p.ws.metric);  // holds the bit planes of the selection keys, not the floats
   int rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, ks.mv, w + p.ws.qsplit, ks.ksplit, false, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, true, true, (int32_t*)(w + p.ws.status), s));
+  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, ks.ksplit, ks.mv, M, true, true, (int32_t*)(w + p.ws.status), s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   rc = cuda_rc(launch_select_planes(p, (const uint32_t*)M, true, idx, cnt, s));
@@ -325,6 +386,7 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   if (!plan || !Q || !K || !V) return STEM_ERR_INVALID_ARG;
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(M)) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
+  if (p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;  // the K side of such a plan lives in the caller's cache
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
@@ -333,7 +395,7 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   float* mv = (float*)(w + p.ws.mv);
   rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, s));
+  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, false, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
   if (M) {
@@ -349,6 +411,7 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
   if (!plan || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
   if (misaligned(M) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3)) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
+  if (!M && p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
@@ -377,11 +440,38 @@ int stem_score_select(const stem_plan* plan, const void* Q, const void* K, const
   if (misaligned(Q) || misaligned(K) || misaligned(V) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3))
     return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
+  if (p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;
   p.last_launches = 0;
-  return enqueue_score_select(p, Q, K, V, w, sel_idx, sel_cnt, (cudaStream_t)stream);
+  return enqueue_score_select(p, Q, K, V, nullptr, w, sel_idx, sel_cnt, (cudaStream_t)stream);
+}
+
+int stem_pool_kv(const stem_plan* plan, const void* K, const void* V, void* kcache, void* stream) {
+  if (!plan || !K || !V || !kcache) return STEM_ERR_INVALID_ARG;
+  if (misaligned(K) || misaligned(V) || ((uintptr_t)kcache & 255)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  if (p.kcache_blocks == 0) return STEM_ERR_INVALID_ARG;
+  const KSide ks = k_side(p, nullptr, kcache);
+  p.last_launches = 0;
+  const int rc = cuda_rc(launch_pool(p, nullptr, K, V, ks.mv, nullptr, ks.ksplit, true, (cudaStream_t)stream));
+  if (rc == STEM_OK) p.last_launches++;
+  return rc;
+}
+
+int stem_score_select_cached(const stem_plan* plan, const void* Q, const void* kcache, int32_t* sel_idx, int32_t* sel_cnt,
+                             void* ws, size_t ws_bytes, void* stream) {
+  if (!plan || !Q || !kcache || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || ((uintptr_t)kcache & 255) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3))
+    return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  if (p.kcache_blocks == 0) return STEM_ERR_INVALID_ARG;
+  int rc = check_ws(p, ws, ws_bytes);
+  if (rc != STEM_OK) return rc;
+  p.last_launches = 0;
+  return enqueue_score_select(p, Q, nullptr, nullptr, const_cast<void*>(kcache), (uint8_t*)ws, sel_idx, sel_cnt,
+                              (cudaStream_t)stream);
 }
 
 int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, const int32_t* sel_idx,
@@ -393,10 +483,31 @@ int stem_sparse_prefill(const stem_plan* plan, const void* Q, const void* K, con
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
   p.last_launches = 0;
-  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, sel_idx, sel_cnt, O, lse, (int32_t*)((uint8_t*)ws + p.ws.status),
-                                       (cudaStream_t)stream));
+  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, sel_idx, sel_cnt, p.share_group, O, lse,
+                                       (int32_t*)((uint8_t*)ws + p.ws.status), (cudaStream_t)stream));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
+}
+
+// Alg. 1 on one stream: steps 1-3c, then step 3d on the lists they wrote.
+static int enqueue_prefill(const Plan& p, const void* Q, const void* K, const void* V, void* O, void* kcache,
+                           bool update_cache, int32_t* sel_idx, int32_t* sel_cnt, float* lse, uint8_t* w, cudaStream_t s) {
+  int32_t* idx = sel_idx ? sel_idx : (int32_t*)(w + p.ws.sel_idx);
+  int32_t* cnt = sel_cnt ? sel_cnt : (int32_t*)(w + p.ws.sel_cnt);
+  p.last_launches = 0;
+  int rc = STEM_OK;
+  if (kcache && update_cache) {
+    const KSide ks = k_side(p, w, kcache);
+    rc = cuda_rc(launch_pool(p, nullptr, K, V, ks.mv, nullptr, ks.ksplit, true, s));
+    if (rc != STEM_OK) return rc;
+    p.last_launches++;
+  }
+  rc = enqueue_score_select(p, Q, kcache ? nullptr : K, kcache ? nullptr : V, kcache, w, idx, cnt, s);
+  if (rc != STEM_OK) return rc;
+  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, idx, cnt, p.share_group, O, lse, (int32_t*)(w + p.ws.status), s));
+  if (rc != STEM_OK) return rc;
+  p.last_launches++;
+  return STEM_OK;
 }
 
 int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, int32_t* sel_idx,
@@ -405,19 +516,23 @@ int stem_prefill(const stem_plan* plan, const void* Q, const void* K, const void
   if ((sel_idx == nullptr) != (sel_cnt == nullptr)) return STEM_ERR_INVALID_ARG;
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
+  if (p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
-  uint8_t* w = (uint8_t*)ws;
-  cudaStream_t s = (cudaStream_t)stream;
-  int32_t* idx = sel_idx ? sel_idx : (int32_t*)(w + p.ws.sel_idx);
-  int32_t* cnt = sel_cnt ? sel_cnt : (int32_t*)(w + p.ws.sel_cnt);
-  p.last_launches = 0;
-  rc = enqueue_score_select(p, Q, K, V, w, idx, cnt, s);
+  return enqueue_prefill(p, Q, K, V, O, nullptr, false, sel_idx, sel_cnt, lse, (uint8_t*)ws, (cudaStream_t)stream);
+}
+
+int stem_prefill_cached(const stem_plan* plan, const void* Q, const void* K, const void* V, void* O, void* kcache,
+                        int update_cache, int32_t* sel_idx, int32_t* sel_cnt, float* lse, void* ws, size_t ws_bytes,
+                        void* stream) {
+  if (!plan || !Q || !K || !V || !O || !kcache) return STEM_ERR_INVALID_ARG;
+  if ((sel_idx == nullptr) != (sel_cnt == nullptr)) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O) || ((uintptr_t)kcache & 255)) return STEM_ERR_INVALID_ARG;
+  const Plan& p = plan->p;
+  if (p.kcache_blocks == 0) return STEM_ERR_INVALID_ARG;
+  int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_sparse_attention(p, Q, K, V, idx, cnt, O, lse, (int32_t*)(w + p.ws.status), s));
-  if (rc != STEM_OK) return rc;
-  p.last_launches++;
-  return STEM_OK;
+  return enqueue_prefill(p, Q, K, V, O, kcache, update_cache != 0, sel_idx, sel_cnt, lse, (uint8_t*)ws, (cudaStream_t)stream);
 }
 
 int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* detail) {

@@ -18,41 +18,56 @@ constexpr int kHeadDim = 128;
 constexpr int kStatusWords = 8;
 constexpr int kRoleSelfTest = 99;  // role recorded by stem_selftest_wait_timeout
 
-// Device-side row tables, built once per plan.
+// Device-side tables, built once per plan.  Query-block rows and key blocks are numbered separately:
+// with chunked prefill the queries are a chunk of every sequence (rows r0 .. N_blk - 1 of it) while the
+// keys are its whole prefix (blocks 0 .. N_blk - 1); without chunks r0 = 0 and the two coincide.
 struct RowTables {
-  const int32_t* row_seq;      // [R_tot] sequence of global row R
-  const int32_t* row_r;        // [R_tot] row index inside its sequence
-  const int32_t* row_tok0;     // [R_tot] first packed token of the row's query block
+  const int32_t* row_seq;      // [R_tot] sequence of query row R
+  const int32_t* row_r;        // [R_tot] row index inside its sequence (global: counts from the sequence's first block)
+  const int32_t* row_tok0;     // [R_tot] first token of the row's query block in the packed Q / O
   const int32_t* row_ntok;     // [R_tot] valid tokens in that block (<= B)
   const int32_t* row_keff;     // [R_tot] budget k_eff(r)
-  const int32_t* seq_tok0;     // [batch] first packed token of the sequence
-  const int32_t* seq_len;      // [batch]
-  const int32_t* seq_nblk;     // [batch]
-  const int32_t* seq_row_off;  // [batch] global row of the sequence's row 0
-  const int64_t* seq_m_off;    // [batch] offset of the sequence's square inside one head of M
+  const int32_t* seq_tok0;     // [batch] first token of the sequence in the packed K / V
+  const int32_t* seq_nblk;     // [batch] key blocks of the sequence (its prefix, with chunks)
+  const int32_t* seq_r0;       // [batch] first row of the query chunk (0 without chunks)
+  const int32_t* seq_row_off;  // [batch] query row R of the chunk's first row
+  const int32_t* seq_kb_off;   // [batch] pooled-K row of the sequence's block 0
+  const int64_t* seq_m_off;    // [batch] offset of the sequence inside one head of M ((N_blk - r0) x N_blk entries)
   const int64_t* seq_mt_off;   // [batch] offset of the sequence inside one head of the bit-plane metric
+  const int32_t* kb_tok0;      // [n_kb_all] first packed K / V token of every key block (sequence-major)
+  const int32_t* kb_ntok;      // [n_kb_all] its valid tokens
+  const int32_t* kb_dst;       // [n_kb_all] its pooled-K row
+  const int32_t* kb_new;       // [n_kb_new] indices into the three arrays above of the blocks that the chunk adds
 };
 
 // Where things live inside the caller's workspace (byte offsets, 256-aligned).
 struct WorkspaceLayout {
   size_t status = 0;
-  size_t mv = 0;       // fp32 [H_kv, R_tot]
-  size_t qsplit = 0;   // bf16 [3, H_q, R_tot, d]: Qbar as hi + mid + lo parts
-  size_t ksplit = 0;   // bf16 [3, H_kv, R_tot, d]: Kbar likewise (row = global block row)
-  size_t metric = 0;   // uint32 [H_q, mt_tot]: the metric of the fused path as bit planes of its selection keys
-  size_t sel_idx = 0;  // int32 [H_q, R_tot, k_max]
-  size_t sel_cnt = 0;  // int32 [H_q, R_tot]
+  size_t mv = 0;       // fp32 [H_kv, KB_tot]
+  size_t qsplit = 0;   // bf16 [3, H_list, R_tot, d]: Qbar as hi + mid + lo parts
+  size_t ksplit = 0;   // bf16 [3, H_kv, KB_tot, d]: Kbar likewise
+  size_t metric = 0;   // uint32 [H_list, mt_tot]: the metric of the fused path as bit planes of its selection keys
+  size_t sel_idx = 0;  // int32 [H_list, R_tot, k_max]
+  size_t sel_cnt = 0;  // int32 [H_list, R_tot]
   size_t total = 0;
 };
 
 struct Plan {
   stem_config cfg{};
-  std::vector<int32_t> cu;  // host copy of cu_seqlens
+  std::vector<int32_t> cu;  // host copy of cu_seqlens (K / V packing)
   int device = 0;
   int sm_count = 0;
-  int32_t T = 0, R_tot = 0, k_max = 0, max_nblk = 0;
+  int32_t T = 0;       // tokens of the packed Q / O
+  int32_t T_kv = 0;    // tokens of the packed K / V
+  int32_t R_tot = 0;   // query rows
+  int32_t KB_tot = 0;  // rows of the pooled K tensors (key blocks; batch x capacity with a caller-owned cache)
+  int32_t n_kb_all = 0, n_kb_new = 0;
+  int32_t k_max = 0, max_nblk = 0;
+  int32_t kcache_blocks = 0;  // per-sequence capacity of a caller-owned pooled-K cache (0: none)
+  bool share_group = false;   // one index list per (kv head, row)
+  int32_t H_list = 0;         // heads of the metric and of the lists: H_q, or H_kv with share_group
   int64_t m_tot = 0;
-  int64_t mt_tot = 0;  // words per head of the bit-plane metric: sum_b N_blk(b) * roundup(N_blk(b), 32)
+  int64_t mt_tot = 0;  // words per head of the bit-plane metric: sum_b rows(b) * roundup(N_blk(b), 32)
   int64_t selected_blocks = 0, causal_blocks = 0, selected_pairs = 0, causal_pairs = 0;
   std::vector<int32_t> k_eff;  // host copy [R_tot]
   float score_scale = 1.f, softmax_scale = 0.f;
@@ -62,7 +77,7 @@ struct Plan {
   RowTables rows{};
   const int32_t* d_gemm_tiles = nullptr;  // [n_gemm_tiles][3] (sequence, row tile, column tile) of the metric GEMM
   int32_t n_gemm_tiles = 0;
-  const int32_t* d_work_sparse = nullptr;  // [n_items][2] (head, global row), attention work order
+  const int32_t* d_work_sparse = nullptr;  // [n_items][2] (head, query row), attention work order
   const int32_t* d_work_dense = nullptr;
   int32_t n_items = 0;
 
@@ -70,10 +85,19 @@ struct Plan {
   mutable int last_launches = 0;
 };
 
+// Byte offsets inside a caller-owned pooled-K cache: Kbar parts bf16 [3, H_kv, KB_tot, d], then MV fp32 [H_kv, KB_tot].
+inline size_t kcache_mv_offset(const Plan& p) {
+  return ((size_t)3 * p.cfg.num_kv_heads * p.KB_tot * kHeadDim * 2 + 255) / 256 * 256;
+}
+inline size_t kcache_bytes(const Plan& p) { return kcache_mv_offset(p) + (size_t)p.cfg.num_kv_heads * p.KB_tot * 4; }
+
 // Kernel launchers (each returns the cudaError_t of the launch).
-// Alg. 1 step 1: mv fp32 [H_kv, R_tot]; qsplit / ksplit bf16 [3, H, R_tot, d], the pooled vectors as hi + mid + lo parts.
+// Alg. 1 step 1.  Q side (Q != null): Qbar of every query row as hi + mid + lo bf16 parts into qsplit
+// [3, H_list, R_tot, d] (the mean over the heads of a kv group as well, with share_group).  K side (K, V != null):
+// Kbar parts into ksplit [3, H_kv, KB_tot, d] and MV into mv [H_kv, KB_tot], for every key block of the plan or,
+// with only_new, for the blocks the chunk adds.
 cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void* V, float* mv, void* qsplit, void* ksplit,
-                        cudaStream_t s);
+                        bool only_new, cudaStream_t s);
 
 // Metric of every causal block (layout of stem_score's M) from the split pooled vectors, on the tensor cores.
 // as_keys: instead of the floats, store bit planes of the selection's order-preserving keys: row r of sequence b at
@@ -92,8 +116,9 @@ cudaError_t launch_select_rows(const Plan& p, const float* M, bool dependent, in
 cudaError_t launch_select_planes(const Plan& p, const uint32_t* Mt, bool dependent, int32_t* sel_idx, int32_t* sel_cnt,
                                  cudaStream_t s);
 
+// list_group: the lists are per kv head ([H_kv, R_tot, k_max]); every query head of a group walks its group's list.
 cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K, const void* V,
-                                    const int32_t* sel_idx, const int32_t* sel_cnt, void* O, float* lse,
+                                    const int32_t* sel_idx, const int32_t* sel_cnt, bool list_group, void* O, float* lse,
                                     int32_t* status, cudaStream_t s);
 
 // One thread waits 1 ms on a barrier nobody arrives at and records the time-out in status words 0..3.

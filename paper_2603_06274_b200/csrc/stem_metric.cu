@@ -57,12 +57,12 @@ constexpr uint32_t kIdesc = make_idesc(kTile, kTile, 0);
 
 struct GemmArgs {
   const int32_t* tiles;  // [n_tiles][3] (sequence, row tile, column tile), column tile <= row tile
-  const float* mv;       // [H_kv, R_tot]
+  const float* mv;       // [H_kv, KB_tot]
   float* M;
   int32_t* status;
   RowTables rows;
   int64_t m_tot, mt_tot;
-  int Hq, Hkv, g, R_tot;
+  int Hq, Hkv, g, R_tot, KB_tot;  // Hq = heads of the metric (the list heads), g = of them per kv head
   float beta, scale;
   int as_keys;  // write bit planes of the metric's selection keys (for launch_select_planes) instead of floats
 };
@@ -82,9 +82,10 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   // accumulators in tensor memory let the epilogue of one head overlap the MMAs of the next.
   const int seq = a.tiles[3 * blockIdx.x], ti = a.tiles[3 * blockIdx.x + 1], tj = a.tiles[3 * blockIdx.x + 2];
   const int kvh = blockIdx.y, g = a.g;
-  const int nb = a.rows.seq_nblk[seq];
-  const int row_off = a.rows.seq_row_off[seq];
-  const int R0 = row_off + ti * kTile, C0 = row_off + tj * kTile;  // first global block row of A and of B
+  const int nb = a.rows.seq_nblk[seq];   // key blocks of the sequence
+  const int r0 = a.rows.seq_r0[seq];     // first row of its query chunk
+  const int R0 = a.rows.seq_row_off[seq] + ti * kTile;  // first query row of A (Qbar numbering)
+  const int C0 = a.rows.seq_kb_off[seq] + tj * kTile;   // first key block of B (Kbar numbering)
 
   if (threadIdx.x == 0) {
     mbar_init(b_full, 1);
@@ -107,7 +108,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   asm volatile("griddepcontrol.wait;" ::: "memory");
   if (threadIdx.x < kTile) {
     const int c = threadIdx.x;  // bias of column c of the tile (the same for every head of the group)
-    bias[c] = (tj * kTile + c < nb) ? a.beta * a.mv[(int64_t)kvh * a.R_tot + C0 + c] : 0.f;
+    bias[c] = (tj * kTile + c < nb) ? a.beta * a.mv[(int64_t)kvh * a.KB_tot + C0 + c] : 0.f;
   }
   tc_fence_before();
   __syncthreads();
@@ -179,7 +180,8 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     // share each quarter of the accumulator rows: warps 0-3 take columns 0-63, warps 4-7 columns 64-127.
     const int quarter = warp & 3, gq0 = (warp >> 2) * 2;
     const int m = quarter * 32 + lane;  // row of the tile == TMEM lane
-    const int r = ti * kTile + m;       // row inside the sequence
+    const int rl = ti * kTile + m;      // row inside the chunk
+    const int r = r0 + rl;              // row inside the sequence
     const int stride = (nb + 31) & ~31;
     float* stage = (float*)(smem_gen + kSmemStage) + warp * 32 * 32;
     bool ok = true;
@@ -190,7 +192,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       if (!ok) break;
       tc_fence_after();
       const uint32_t taddr = tmem + (uint32_t)(hh & 1) * 128u + ((uint32_t)(quarter * 32) << 16);
-      uint32_t* dst_planes = (uint32_t*)a.M + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)r * stride + tj * kTile;
+      uint32_t* dst_planes = (uint32_t*)a.M + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)rl * stride + tj * kTile;
       float* mseq = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq];
 #pragma unroll 1
       for (int gq = gq0; gq < gq0 + 2; ++gq) {
@@ -237,9 +239,9 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           __syncwarp();
           const int cg = tj * kTile + gq * 32 + lane;  // this lane's column inside the sequence
           for (int mm = 0; mm < 32; ++mm) {
-            const int rr = ti * kTile + quarter * 32 + mm;
+            const int rr = r0 + ti * kTile + quarter * 32 + mm;  // row inside the sequence
             if (rr >= nb) break;
-            if (cg <= rr) mseq[(int64_t)rr * nb + cg] = stage[mm * 32 + (((lane >> 2) ^ (mm & 7)) << 2) + (lane & 3)];
+            if (cg <= rr) mseq[(int64_t)(rr - r0) * nb + cg] = stage[mm * 32 + (((lane >> 2) ^ (mm & 7)) << 2) + (lane & 3)];
           }
           __syncwarp();
         }
@@ -266,13 +268,13 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t planes) 
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
                                bool as_keys, bool dependent, int32_t* status, cudaStream_t s) {
   CUtensorMap mq, mk;
-  if (!make_map(&mq, qsplit, p.R_tot, 3 * (int64_t)p.cfg.num_q_heads) ||
-      !make_map(&mk, ksplit, p.R_tot, 3 * (int64_t)p.cfg.num_kv_heads))
+  if (!make_map(&mq, qsplit, p.R_tot, 3 * (int64_t)p.H_list) ||
+      !make_map(&mk, ksplit, p.KB_tot, 3 * (int64_t)p.cfg.num_kv_heads))
     return cudaErrorInvalidValue;
   GemmArgs a{};
   (void)status;
   a.tiles = p.d_gemm_tiles; a.mv = mv; a.M = M; a.status = status; a.rows = p.rows; a.m_tot = p.m_tot; a.mt_tot = p.mt_tot;
-  a.Hq = p.cfg.num_q_heads; a.Hkv = p.cfg.num_kv_heads; a.g = a.Hq / a.Hkv; a.R_tot = p.R_tot;
+  a.Hq = p.H_list; a.Hkv = p.cfg.num_kv_heads; a.g = a.Hq / a.Hkv; a.R_tot = p.R_tot; a.KB_tot = p.KB_tot;
   a.beta = p.cfg.beta; a.scale = p.score_scale; a.as_keys = as_keys ? 1 : 0;
   // the attribute belongs to the device's context: set it once per device of this process
   static bool attr_set[64] = {};

@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_rows_kerne
   const int n_forced = i - n_cand;
   const int need = max(min(a.rows.row_keff[R] - n_forced, n_cand), 0);
   int32_t* out = a.sel_idx + ((int64_t)h * a.R_tot + R) * a.k_max;
-  const float* mrow = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq] + (int64_t)r * nb + c_lo;
+  const float* mrow = a.M + (int64_t)h * a.m_tot + a.rows.seq_m_off[seq] + (int64_t)(r - a.rows.seq_r0[seq]) * nb + c_lo;
   const int per = (n_cand + 31) >> 5;  // candidates per lane
 
   uint32_t sel[SETS];  // per key of this lane (bit t <-> its t-th candidate): selected
@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, SETS == 1 ? 4 : 2) select_planes_ker
   const int need = max(min(a.rows.row_keff[R] - n_forced, n_cand), 0);
   int32_t* out = a.sel_idx + ((int64_t)h * a.R_tot + R) * a.k_max;
   const int stride = (nb + 31) & ~31;
-  const uint32_t* prow = a.Mt + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)r * stride;
+  const uint32_t* prow = a.Mt + (int64_t)h * a.mt_tot + a.rows.seq_mt_off[seq] + (int64_t)(r - a.rows.seq_r0[seq]) * stride;
 
   uint32_t sel[SETS];
 #pragma unroll
@@ -308,7 +308,7 @@ int row_select_max_blocks() { return 2 * 1024; }
 static SelArgs make_args(const Plan& p, int32_t* sel_idx, int32_t* sel_cnt) {
   SelArgs a{};
   a.sel_idx = sel_idx; a.sel_cnt = sel_cnt; a.rows = p.rows; a.m_tot = p.m_tot; a.mt_tot = p.mt_tot;
-  a.Hq = p.cfg.num_q_heads; a.R_tot = p.R_tot; a.k_max = p.k_max;
+  a.Hq = p.H_list; a.R_tot = p.R_tot; a.k_max = p.k_max;
   a.stem = p.cfg.stem_blocks; a.local = p.cfg.local_blocks;
   return a;
 }

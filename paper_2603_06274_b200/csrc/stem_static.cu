@@ -54,12 +54,13 @@ extern "C" int stem_score_static(const stem_plan* plan, const void* Q, const voi
   if (!plan || !Q || !K || !V || !M) return STEM_ERR_INVALID_ARG;
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)M) & 15) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
+  if (p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
 
   // Size check first: nothing is touched when the problem does not fit.
   const size_t status_bytes = align256(kStatusWords * sizeof(int32_t));
-  const size_t mv_bytes = align256((size_t)p.cfg.num_kv_heads * p.R_tot * sizeof(float));
-  const size_t q_bytes = align256((size_t)3 * p.cfg.num_q_heads * p.R_tot * kHeadDim * 2);
-  const size_t k_bytes = align256((size_t)3 * p.cfg.num_kv_heads * p.R_tot * kHeadDim * 2);
+  const size_t mv_bytes = align256((size_t)p.cfg.num_kv_heads * p.KB_tot * sizeof(float));
+  const size_t q_bytes = align256((size_t)3 * p.H_list * p.R_tot * kHeadDim * 2);
+  const size_t k_bytes = align256((size_t)3 * p.cfg.num_kv_heads * p.KB_tot * kHeadDim * 2);
   if (status_bytes + mv_bytes + q_bytes + k_bytes > (size_t)STEM_STATIC_SCRATCH_BYTES) return STEM_ERR_STATIC_SCRATCH;
 
   int device = -1;
@@ -81,7 +82,7 @@ extern "C" int stem_score_static(const stem_plan* plan, const void* Q, const voi
   // (tiles that reach past a sequence's last block read rows of a neighbour or stale rows, and only
   // into entries the epilogue never stores).
   if (cudaMemsetAsync(status, 0, kStatusWords * sizeof(int32_t), s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
-  if (launch_pool(p, Q, K, V, mv, qsplit, ksplit, s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  if (launch_pool(p, Q, K, V, mv, qsplit, ksplit, false, s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   p.last_launches++;
   if (launch_metric_gemm(p, qsplit, ksplit, mv, M, false, true, status, s) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
   p.last_launches++;
