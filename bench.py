@@ -363,6 +363,7 @@ def main():
         res["selected_blocks"] = int(info.selected_blocks)
         res["causal_blocks"] = int(info.causal_blocks)
         if extras:
+            fused_out = out.clone()     # the dense comparator below overwrites `out`
             dsteps = max(2, min(steps, 3))
             res["dense_ms"] = time_loop(lambda: pkg.stem_sparse_prefill(plan, q, k, v, None, None, out), dsteps, 1)[0]
             # end to end with HOST buffers: H2D of Q, K, V and D2H of O inside the timed region, every step
@@ -370,8 +371,9 @@ def main():
             pipe = GroupPipeline(w, data)
             res["e2e_ms"] = time_loop(pipe.step, max(2, min(steps, 5)), 2)[0]
             pipe.check()
-            res["e2e_identical"] = bool(torch.equal(torch.cat([o.view(torch.int16) for o in pipe.o], dim=1), out.view(torch.int16))
-                                        and torch.equal(pipe.ho.cuda(), out.view(torch.int16)))
+            res["e2e_identical"] = bool(torch.equal(torch.cat([o.view(torch.int16) for o in pipe.o], dim=1), fused_out.view(torch.int16))
+                                        and torch.equal(pipe.ho.cuda(), fused_out.view(torch.int16)))
+            del fused_out
             res["e2e_launches_per_step"] = pipe.launches
             res["h2d"], res["d2h"] = int(pipe.h2d), int(pipe.d2h)
             pipe.close()

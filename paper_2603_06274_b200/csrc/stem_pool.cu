@@ -45,7 +45,7 @@ struct PoolArgs {
   __nv_bfloat16 *qsplit, *ksplit;
 };
 
-template <int kBlock>
+template <int kBlock, bool kGroupMean>
 __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
   constexpr int kTokPerWarp = kBlock / 4;
   constexpr int kSteps = kTokPerWarp / 2;
@@ -80,13 +80,28 @@ __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
     dst_row = a.rows.kb_dst[kb];
   }
 
+  // every load of the block (of its first head) is issued before anything else happens
+  uint4 raw[kSteps];
+#pragma unroll
+  for (int i = 0; i < kSteps; ++i) {
+    const int t = warp * kTokPerWarp + 2 * i + half;
+    raw[i] = make_uint4(0, 0, 0, 0);
+    if (t < ntok) raw[i] = ld_stream(base + (int64_t)(tok0 + t) * st + chunk * 8);
+  }
+
   __shared__ float red[4][kHeadDim];
   __shared__ float redmax[4];
 
   if (kind < 2) {
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    for (int hh = 0; hh < n_heads; ++hh) {
-      uint4 raw[kSteps];
+#pragma unroll
+    for (int i = 0; i < kSteps; ++i) {
+      float f[8];
+      unpack8(raw[i], f);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) acc[c] += f[c];
+    }
+    for (int hh = 1; kGroupMean && hh < n_heads; ++hh) {  // the other query heads of the group (one list per kv head)
 #pragma unroll
       for (int i = 0; i < kSteps; ++i) {
         const int t = warp * kTokPerWarp + 2 * i + half;
@@ -125,13 +140,6 @@ __global__ void __launch_bounds__(128) pool_kernel(const PoolArgs a) {
     dst[at + plane] = mid;
     dst[at + 2 * plane] = lo;
   } else {
-    uint4 raw[kSteps];
-#pragma unroll
-    for (int i = 0; i < kSteps; ++i) {
-      const int t = warp * kTokPerWarp + 2 * i + half;
-      raw[i] = make_uint4(0, 0, 0, 0);
-      if (t < ntok) raw[i] = ld_stream(base + (int64_t)(tok0 + t) * st + chunk * 8);
-    }
     float best = 0.f;  // squared norms are >= 0
 #pragma unroll
     for (int i = 0; i < kSteps; ++i) {
@@ -171,8 +179,14 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
   const int64_t n_k = K ? (int64_t)(only_new ? p.n_kb_new : p.n_kb_all) * 2 * p.cfg.num_kv_heads : 0;
   const dim3 grid((unsigned)(a.n_q + n_k));
   if (grid.x == 0) return cudaSuccess;
-  if (p.cfg.block == 128) pool_kernel<128><<<grid, 128, 0, s>>>(a);
-  else pool_kernel<64><<<grid, 128, 0, s>>>(a);
+  const bool group_mean = a.heads_per_list > 1;
+  if (p.cfg.block == 128) {
+    if (group_mean) pool_kernel<128, true><<<grid, 128, 0, s>>>(a);
+    else pool_kernel<128, false><<<grid, 128, 0, s>>>(a);
+  } else {
+    if (group_mean) pool_kernel<64, true><<<grid, 128, 0, s>>>(a);
+    else pool_kernel<64, false><<<grid, 128, 0, s>>>(a);
+  }
   return cudaGetLastError();
 }
 
