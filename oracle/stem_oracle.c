@@ -28,6 +28,8 @@
  * Chunked prefill (so_*_chunk) is pinned against the one-shot functions: the rows of any split of a
  * sequence into chunks must reproduce the one-shot lists bit for bit and the outputs to 1e-6; the
  * group-shared metric (so_metric_shared) against a numpy fp64 mean of per-head metrics.
+ * The anti-diagonal scoring mode (so_metric_antidiag) is pinned against the anti-diagonal of a numpy fp64
+ * score matrix and against hand-built inputs whose anti-diagonal sums are known in closed form.
  * End-task accuracy (the paper's tables) needs trained weights: parity unpinned.
  *
  * Layouts
@@ -528,6 +530,59 @@ void so_metric_shared(const float* qbar /*[Hq,R_tot,d]*/, const float* kbar /*[H
                     }
                     double m = (double)score_scale * (sum / (double)g) + (double)beta * (double)mv[(int64_t)kvh * r_tot + row_off + j];
                     Mg[(int64_t)kvh * m_tot + m_off + r * nb + j] = (float)m;
+                }
+            }
+        }
+        row_off += nb;
+        m_off += nb * nb;
+    }
+}
+
+/* =============================================================================================
+ * Anti-diagonal scoring (Overall Algorithm: the pooling step is called anti-diagonal scoring, after
+ * XAttention; Alg. 1 step 1 comment "Pool(Q, K, stride = B)").  The other reading of the pooling
+ * step: instead of the product of block means, the routing term of block pair (r, j) is the mean
+ * of the token scores ALONG THE MAIN ANTI-DIAGONAL of the B x B score block (stride B leaves one
+ * anti-diagonal per block),
+ *   A[h,r,j] = (1/n) * sum_{s=0..B-1, both tokens exist} q[rB + B-1-s] . k[jB + s],
+ * n = number of such s (B for full blocks), and M = score_scale * A + beta * MV as in Eq. 7.
+ * Layout of M as in so_metric.
+ * =========================================================================================== */
+void so_metric_antidiag(const uint16_t* Q, int64_t q_stride_tok, int64_t q_stride_head, const uint16_t* K,
+                        int64_t kv_stride_tok, int64_t kv_stride_head, const float* mv /*[Hkv,R_tot]*/, int32_t Hq,
+                        int32_t Hkv, int32_t d, int32_t batch, const int32_t* cu_seqlens, int32_t B, float beta,
+                        float score_scale, float* M /*[Hq,m_tot]*/) {
+    int64_t r_tot = 0, m_tot = 0;
+    for (int b = 0; b < batch; ++b) {
+        int64_t nb = cdiv(cu_seqlens[b + 1] - cu_seqlens[b], B);
+        r_tot += nb;
+        m_tot += nb * nb;
+    }
+    int g = Hq / Hkv;
+    int64_t row_off = 0, m_off = 0;
+    for (int b = 0; b < batch; ++b) {
+        int64_t t0 = cu_seqlens[b], n = cu_seqlens[b + 1] - cu_seqlens[b];
+        int64_t nb = cdiv(n, B);
+#pragma omp parallel for collapse(2) schedule(dynamic, 4)
+        for (int h = 0; h < Hq; ++h) {
+            for (int64_t r = 0; r < nb; ++r) {
+                int kvh = h / g;
+                for (int64_t j = 0; j <= r; ++j) {
+                    double acc = 0.0;
+                    int64_t pairs = 0;
+                    for (int64_t s = 0; s < B; ++s) {
+                        int64_t tq = r * B + (B - 1 - s), tk = j * B + s;
+                        if (tq >= n || tk >= n) continue;
+                        const uint16_t* qp = Q + (t0 + tq) * q_stride_tok + (int64_t)h * q_stride_head;
+                        const uint16_t* kp = K + (t0 + tk) * kv_stride_tok + (int64_t)kvh * kv_stride_head;
+                        double dot = 0.0;
+                        for (int c = 0; c < d; ++c) dot += (double)bf16_to_f32(qp[c]) * (double)bf16_to_f32(kp[c]);
+                        acc += dot;
+                        ++pairs;
+                    }
+                    double a = pairs > 0 ? acc / (double)pairs : 0.0;
+                    double m = (double)score_scale * a + (double)beta * (double)mv[(int64_t)kvh * r_tot + row_off + j];
+                    M[(int64_t)h * m_tot + m_off + r * nb + j] = (float)m;
                 }
             }
         }

@@ -356,3 +356,32 @@ def metric_shared(qbar: np.ndarray, kbar: np.ndarray, mv: np.ndarray, nblk: np.n
 def expand_group_lists(idx_g: np.ndarray, cnt_g: np.ndarray, g: int):
     """Per-kv-head lists [H_kv, R, k] -> per-query-head lists [H_kv * g, R, k] (every head of a group gets its list)."""
     return np.repeat(idx_g, g, axis=0), np.repeat(cnt_g, g, axis=0)
+
+
+# ----------------------------------------------------------------------------------------------
+# Anti-diagonal scoring mode (Overall Algorithm; Alg. 1 step 1 comment)
+# ----------------------------------------------------------------------------------------------
+
+def metric_antidiag(q_bits: np.ndarray, k_bits: np.ndarray, mv: np.ndarray, cu_seqlens: np.ndarray, block: int,
+                    beta: float, score_scale: float = 1.0) -> np.ndarray:
+    """Metric with the routing term taken as the mean of the token scores along the main anti-diagonal of every
+    B x B score block -> fp32 [H_q, sum_b N_blk_b^2] (entries j <= r defined, rest NaN)."""
+    T, hq, d = q_bits.shape
+    hkv = k_bits.shape[1]
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    nblk = n_blocks(np.diff(cu), block)
+    m_tot = int((nblk.astype(np.int64) ** 2).sum())
+    M = np.full((hq, m_tot), np.nan, dtype=np.float32)
+    qs, qh = _strides(q_bits)
+    ks, kh = _strides(k_bits)
+    _load().so_metric_antidiag(_p(q_bits), ctypes.c_int64(qs), ctypes.c_int64(qh), _p(k_bits), ctypes.c_int64(ks),
+                               ctypes.c_int64(kh), _p(np.ascontiguousarray(mv, dtype=np.float32)), ctypes.c_int32(hq),
+                               ctypes.c_int32(hkv), ctypes.c_int32(d), ctypes.c_int32(len(cu) - 1), _p(cu),
+                               ctypes.c_int32(block), ctypes.c_float(beta), ctypes.c_float(score_scale), _p(M))
+    return M
+
+
+def score_antidiag(q_bits, k_bits, v_bits, cu_seqlens, p: StemParams):
+    """Steps 1 and 3a in the anti-diagonal scoring mode. Returns (M, mv)."""
+    mv = value_magnitude(v_bits, cu_seqlens, p.block)
+    return metric_antidiag(q_bits, k_bits, mv, cu_seqlens, p.block, p.beta, p.score_scale), mv

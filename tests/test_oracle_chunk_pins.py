@@ -139,3 +139,46 @@ def test_group_metric_is_the_mean_of_the_heads_metrics():
     M1, qb1, kb1, mv1 = so.score(d1["q"], d1["k"], d1["v"], d1["cu_seqlens"], p1)
     Mg1 = so.metric_shared(qb1, kb1, mv1, so.n_blocks(w1.seqlens, 64), p1.beta, p1.score_scale)
     assert np.array_equal(np.nan_to_num(M1, nan=-7.0), np.nan_to_num(Mg1, nan=-7.0))
+
+
+def test_antidiagonal_metric_is_the_mean_of_the_blocks_main_antidiagonal():
+    """Anti-diagonal scoring mode (Overall Algorithm; Alg. 1 step 1 comment, stride = B): pinned against the
+    anti-diagonal of a numpy fp64 score matrix, and on inputs whose anti-diagonal sums have a closed form."""
+    w = wl.small("antidiag", seqlens=(700, 200), hq=4, hkv=2, block=64, permille=300)
+    data = wl.make_qkv(w)
+    p = oracle_params(w)
+    M, mv = so.score_antidiag(data["q"], data["k"], data["v"], data["cu_seqlens"], p)
+    B, cu, g = w.block, data["cu_seqlens"], 2
+    q = wl.bf16_bits_to_f32(data["q"]).astype(np.float64)
+    k = wl.bf16_bits_to_f32(data["k"]).astype(np.float64)
+    nblk = so.n_blocks(w.seqlens, B)
+    row_off = np.concatenate([[0], np.cumsum(nblk)])
+    off = 0
+    for b, nb in enumerate(nblk):
+        nb, n = int(nb), w.seqlens[b]
+        for h in range(w.num_q_heads):
+            S = q[cu[b]:cu[b + 1], h] @ k[cu[b]:cu[b + 1], h // g].T          # every token score of the sequence
+            Sp = np.full((nb * B, nb * B), np.nan)
+            Sp[:n, :n] = S
+            got = M[h, off:off + nb * nb].reshape(nb, nb)
+            for r in range(nb):
+                for j in range(r + 1):
+                    blk = Sp[r * B:(r + 1) * B, j * B:(j + 1) * B]
+                    anti = np.array([blk[B - 1 - s, s] for s in range(B)])     # main anti-diagonal
+                    a = np.nanmean(anti) if np.isfinite(anti).any() else 0.0  # no existing pair: the term is 0
+                    want = p.score_scale * a + p.beta * mv[h // g, row_off[b] + j]
+                    assert abs(got[r, j] - want) <= 1e-6 * max(1.0, abs(want))
+                assert np.isnan(got[r, r + 1:]).all()
+        off += nb * nb
+    # closed form: q_t = a_t * u, k_t = c_t * u with |u| = 1  =>  the anti-diagonal mean of block (r, j) is
+    # mean_s a[rB + B-1-s] * c[jB + s]; with a_t = t + 1 and c_t = 1 that is the mean position of the query block
+    n, B, d = 256, 64, 128
+    u = np.zeros(d, np.float32); u[3] = 1.0
+    qf = (np.arange(1, n + 1, dtype=np.float32)[:, None] * u[None, :])[:, None, :]
+    kf = np.broadcast_to(u, (n, 1, d)).astype(np.float32)
+    vf = np.zeros((n, 1, d), np.float32)
+    cu1 = np.array([0, n], np.int32)
+    mv0 = so.value_magnitude(wl.f32_to_bf16_bits(vf), cu1, B)
+    M2 = so.metric_antidiag(wl.f32_to_bf16_bits(qf), wl.f32_to_bf16_bits(kf), mv0, cu1, B, beta=0.2).reshape(4, 4)
+    for r in range(4):
+        assert np.allclose(M2[r, :r + 1], r * B + (B + 1) / 2.0)
