@@ -120,7 +120,15 @@ typedef struct {
  * share_group (Main Results: integration with a block-level top-k shared by the heads of a GQA group): one
  * index list per (kv head, row).  The group's metric is the mean over its query heads of Eq. 7, i.e. Eq. 7 on
  * the group-mean pooled query; sel_idx / sel_cnt / M have num_kv_heads heads; every query head of the group
- * attends over its group's list. */
+ * attends over its group's list.
+ *
+ * score_mode = 1, anti-diagonal scoring (Overall Algorithm: "anti-diagonal scoring", after XAttention; Alg. 1
+ * step 1 comment, stride = B): the other reading of the pooling step.  The routing term of block pair (r, j)
+ * is the mean of the token scores along the main anti-diagonal of the B x B score block,
+ *   (1/n) sum_s q[rB + B-1-s] . k[jB + s]  over the s whose two tokens exist (n = B for full blocks),
+ * in place of Qbar[h,r] . Kbar[kv(h),j]; the magnitude term, the budget and the selection are unchanged.
+ * Computed as one tensor-core contraction of Q with K (inner dimension B * d).  Not combinable with the
+ * pooled-K cache or share_group; at most 8 sequences per plan (STEM_ERR_UNSUPPORTED otherwise). */
 typedef struct {
   const int32_t* q_start_host;    /* HOST [batch]: first query token of every sequence's chunk, a multiple of
                                      block, < kv_len(b); NULL = 0 (no chunking)                               */
@@ -128,7 +136,8 @@ typedef struct {
                                      NULL = kv_len(b)                                                         */
   int32_t kcache_blocks_per_seq;  /* capacity (blocks per sequence) of a caller-owned pooled-K cache; 0 = none */
   int32_t share_group;            /* 1: one index list per kv head                                            */
-  int32_t reserved[4];            /* must be 0                                                                */
+  int32_t score_mode;             /* 0: product of block means (Eq. 7 on pooled blocks); 1: anti-diagonal scoring */
+  int32_t reserved[3];            /* must be 0                                                                */
 } stem_options;
 
 /* Builds the per-row budget table k_eff(r) (Eq. 3 in block units, i = r+1, clamped by the forced
@@ -250,7 +259,7 @@ int stem_prefill_cached(const stem_plan* plan, const void* Q, const void* K, con
  * Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in a kernel gave up; outputs of that
  * call are undefined) or STEM_ERR_CUDA.  detail (optional, HOST int32[4]) receives the raw words:
  * {1, CTA index, role, barrier id} of the attention kernel, or {2, tile, kv head, 0} when
- * the wait that gave up was in the metric kernel. */
+ * the wait that gave up was in the metric kernel ({3, tile, query head, 0}: its anti-diagonal form). */
 int stem_check_status(const stem_plan* plan, void* workspace, void* stream, int32_t* detail_host);
 
 /* Self-test of the time-out reporting (the paper has no counterpart).  Enqueues a one-thread kernel

@@ -79,7 +79,8 @@ class StemOptions(ctypes.Structure):
         ("total_len_host", ctypes.POINTER(ctypes.c_int32)),
         ("kcache_blocks_per_seq", ctypes.c_int32),
         ("share_group", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 4),
+        ("score_mode", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 3),
     ]
 
 
@@ -160,11 +161,12 @@ class StemPlan:
                  local_blocks: int = 4, min_blocks: int = 0, beta: float = 0.2, score_scale: float = 0.0,
                  softmax_scale: float = 0.0, head_dim: int = 128, q_strides=None, kv_strides=None,
                  q_starts: Optional[Sequence[int]] = None, total_lens: Optional[Sequence[int]] = None,
-                 kcache_blocks_per_seq: int = 0, share_group: bool = False):
+                 kcache_blocks_per_seq: int = 0, share_group: bool = False, score_mode: int = 0):
         """``seqlens`` are the lengths of K and V.  With ``q_starts`` (chunked prefill) Q and O hold only the
         tokens q_start(b) .. seqlens[b]-1 of every sequence and ``total_lens`` are the full sequence lengths the
         budget schedule is evaluated on; ``kcache_blocks_per_seq`` > 0 puts the pooled K-side tensors into a
-        caller-owned cache (``stem_pool_kv`` / ``*_cached``); ``share_group`` selects one list per kv head."""
+        caller-owned cache (``stem_pool_kv`` / ``*_cached``); ``share_group`` selects one list per kv head;
+        ``score_mode`` = 1 the anti-diagonal scoring mode."""
         lib = load()
         cu = [0]
         for n in seqlens:
@@ -193,6 +195,7 @@ class StemPlan:
             opts.total_len_host = ctypes.cast(self._tl, ctypes.POINTER(ctypes.c_int32))
         opts.kcache_blocks_per_seq = int(kcache_blocks_per_seq)
         opts.share_group = 1 if share_group else 0
+        opts.score_mode = int(score_mode)
         _check(lib.stem_plan_create_ex(ctypes.byref(cfg), ctypes.byref(opts), ctypes.byref(self._h)), "stem_plan_create_ex")
         info = StemPlanInfo()
         _check(lib.stem_plan_query(self._h, ctypes.byref(info)), "stem_plan_query")

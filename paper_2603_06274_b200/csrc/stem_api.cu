@@ -101,9 +101,14 @@ int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_p
   if (rc != STEM_OK) return rc;
   stem_options o{};
   if (opts) o = *opts;
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < 3; ++i)
     if (o.reserved[i] != 0) return STEM_ERR_INVALID_ARG;
   if (o.kcache_blocks_per_seq < 0 || (o.share_group != 0 && o.share_group != 1)) return STEM_ERR_INVALID_ARG;
+  if (o.score_mode != 0 && o.score_mode != 1) return STEM_ERR_INVALID_ARG;
+  // anti-diagonal scoring contracts Q with K directly: no pooled-K cache to read instead, one list per query head,
+  // and one tensor map per sequence (a bounded number of them ride in the kernel's parameters)
+  if (o.score_mode == 1 && (o.kcache_blocks_per_seq > 0 || o.share_group != 0 || cfg->batch > antidiag_max_sequences()))
+    return STEM_ERR_UNSUPPORTED;
   const int B = cfg->block, batch = cfg->batch, Hq = cfg->num_q_heads, Hkv = cfg->num_kv_heads;
   for (int b = 0; b < batch; ++b) {
     const int64_t kv_len = cfg->cu_seqlens_host[b + 1] - cfg->cu_seqlens_host[b];
@@ -123,13 +128,14 @@ int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_p
   p.softmax_scale = cfg->softmax_scale == 0.f ? 1.f / std::sqrt((float)kHeadDim) : cfg->softmax_scale;
   p.kcache_blocks = o.kcache_blocks_per_seq;
   p.share_group = o.share_group != 0;
+  p.score_mode = o.score_mode;
   p.H_list = p.share_group ? Hkv : Hq;
 
   const int g = Hq / Hkv;
   p.T_kv = p.cu[batch];
 
   std::vector<int32_t> row_seq, row_r, row_tok0, row_ntok, seq_tok0(batch), seq_nblk(batch), seq_r0(batch),
-      seq_row_off(batch), seq_kb_off(batch), kb_tok0, kb_ntok, kb_dst, kb_new;
+      seq_row_off(batch), seq_kb_off(batch), seq_kb_first(batch), kb_tok0, kb_ntok, kb_dst, kb_new;
   std::vector<int64_t> seq_m_off(batch), seq_mt_off(batch);
   int64_t m_off = 0, mt_off = 0;
   int32_t q_tok = 0, kb_off = 0;
@@ -145,6 +151,9 @@ int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_p
     seq_r0[b] = r0;
     seq_row_off[b] = (int32_t)row_seq.size();
     seq_kb_off[b] = p.kcache_blocks > 0 ? b * p.kcache_blocks : kb_off;
+    seq_kb_first[b] = (int32_t)kb_tok0.size();
+    p.h_seq_r0.push_back(r0);
+    p.h_seq_qtok0.push_back(q_tok);
     seq_m_off[b] = m_off;
     seq_mt_off[b] = mt_off;
     mt_off += (int64_t)(nb - r0) * ((nb + 31) / 32 * 32);  // rows padded to whole 32-column groups
@@ -251,7 +260,7 @@ int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_p
   const size_t o_row_seq = push(blob, row_seq), o_row_r = push(blob, row_r), o_row_tok0 = push(blob, row_tok0),
                o_row_ntok = push(blob, row_ntok), o_keff = push(blob, p.k_eff), o_seq_tok0 = push(blob, seq_tok0),
                o_seq_nblk = push(blob, seq_nblk), o_seq_r0 = push(blob, seq_r0), o_seq_row_off = push(blob, seq_row_off),
-               o_seq_kb_off = push(blob, seq_kb_off), o_seq_m_off = push(blob, seq_m_off),
+               o_seq_kb_off = push(blob, seq_kb_off), o_seq_kb_first = push(blob, seq_kb_first), o_seq_m_off = push(blob, seq_m_off),
                o_seq_mt_off = push(blob, seq_mt_off), o_kb_tok0 = push(blob, kb_tok0), o_kb_ntok = push(blob, kb_ntok),
                o_kb_dst = push(blob, kb_dst), o_kb_new = push(blob, kb_new), o_gt = push(blob, gemm_tiles),
                o_ws = push(blob, work_sparse), o_wd = push(blob, work_dense);
@@ -273,6 +282,7 @@ int stem_plan_create_ex(const stem_config* cfg, const stem_options* opts, stem_p
   p.rows.seq_r0 = (const int32_t*)(d + o_seq_r0);
   p.rows.seq_row_off = (const int32_t*)(d + o_seq_row_off);
   p.rows.seq_kb_off = (const int32_t*)(d + o_seq_kb_off);
+  p.rows.seq_kb_first = (const int32_t*)(d + o_seq_kb_first);
   p.rows.seq_m_off = (const int64_t*)(d + o_seq_m_off);
   p.rows.seq_mt_off = (const int64_t*)(d + o_seq_mt_off);
   p.rows.kb_tok0 = (const int32_t*)(d + o_kb_tok0);
@@ -358,6 +368,22 @@ static KSide k_side(const Plan& p, uint8_t* w, void* kcache) {
   return {w + p.ws.ksplit, (float*)(w + p.ws.mv)};
 }
 
+// Alg. 1 step 3a from what step 1 left: the product of block means on the pooled vectors, or, in the anti-diagonal
+// scoring mode, the contraction of Q with K itself (MV comes from the pooling kernel in both).
+static int enqueue_metric(const Plan& p, const void* Q, const void* K, uint8_t* w, const KSide& ks, float* M, bool as_keys,
+                          bool dependent, cudaStream_t s) {
+  int32_t* status = (int32_t*)(w + p.ws.status);
+  if (p.score_mode == 1) {
+    int launched = 0;
+    const int rc = cuda_rc(launch_antidiag_metric(p, Q, K, ks.mv, M, as_keys, status, &launched, s));
+    p.last_launches += launched;
+    return rc;
+  }
+  const int rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, ks.ksplit, ks.mv, M, as_keys, dependent, status, s));
+  if (rc == STEM_OK) p.last_launches++;
+  return rc;
+}
+
 // Alg. 1 steps 1-3c on one stream: pooling (one pass over Q and, unless the K side comes from a cache, over K
 // and V; emits the pooled vectors as bf16 parts), the metric of every causal block on the tensor cores into
 // the workspace (stored as bit planes of the selection's order-preserving keys), and the row-wise selection
@@ -370,13 +396,13 @@ static int enqueue_score_select(const Plan& p, const void* Q, const void* K, con
   float* M = (float*)(w + p.ws.metric);  // holds the bit planes of the selection keys, not the floats
   int rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, ks.mv, w + p.ws.qsplit, ks.ksplit, false, s));
+  // (the anti-diagonal mode has no use for the pooled query vectors)
+  rc = cuda_rc(launch_pool(p, p.score_mode == 1 ? nullptr : Q, K, V, ks.mv, w + p.ws.qsplit, ks.ksplit, false, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, ks.ksplit, ks.mv, M, true, true, (int32_t*)(w + p.ws.status), s));
+  rc = enqueue_metric(p, Q, K, w, ks, M, true, true, s);
   if (rc != STEM_OK) return rc;
-  p.last_launches++;
-  rc = cuda_rc(launch_select_planes(p, (const uint32_t*)M, true, idx, cnt, s));
+  rc = cuda_rc(launch_select_planes(p, (const uint32_t*)M, p.score_mode != 1, idx, cnt, s));
   if (rc == STEM_OK) p.last_launches++;
   return rc;
 }
@@ -395,15 +421,11 @@ int stem_score(const stem_plan* plan, const void* Q, const void* K, const void* 
   float* mv = (float*)(w + p.ws.mv);
   rc = cuda_rc(cudaMemsetAsync(w + p.ws.status + 16, 0, 16, s));  // the metric kernel's status words
   if (rc != STEM_OK) return rc;
-  rc = cuda_rc(launch_pool(p, Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, false, s));
+  rc = cuda_rc(launch_pool(p, p.score_mode == 1 ? nullptr : Q, K, V, mv, w + p.ws.qsplit, w + p.ws.ksplit, false, s));
   if (rc != STEM_OK) return rc;
   p.last_launches++;
-  if (M) {
-    rc = cuda_rc(launch_metric_gemm(p, w + p.ws.qsplit, w + p.ws.ksplit, mv, M, false, true, (int32_t*)(w + p.ws.status), s));
-    if (rc != STEM_OK) return rc;
-    p.last_launches++;
-  }
-  return STEM_OK;
+  if (M) rc = enqueue_metric(p, Q, K, w, k_side(p, w, nullptr), M, false, true, s);
+  return rc;
 }
 
 int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t* sel_cnt, void* ws, size_t ws_bytes,
@@ -411,7 +433,7 @@ int stem_select(const stem_plan* plan, const float* M, int32_t* sel_idx, int32_t
   if (!plan || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
   if (misaligned(M) || ((uintptr_t)sel_idx & 3) || ((uintptr_t)sel_cnt & 3)) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
-  if (!M && p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
+  if (!M && (p.kcache_blocks > 0 || p.score_mode == 1)) return STEM_ERR_INVALID_ARG;  // nothing pooled to recompute M from
   int rc = check_ws(p, ws, ws_bytes);
   if (rc != STEM_OK) return rc;
   uint8_t* w = (uint8_t*)ws;

@@ -32,6 +32,7 @@ struct RowTables {
   const int32_t* seq_r0;       // [batch] first row of the query chunk (0 without chunks)
   const int32_t* seq_row_off;  // [batch] query row R of the chunk's first row
   const int32_t* seq_kb_off;   // [batch] pooled-K row of the sequence's block 0
+  const int32_t* seq_kb_first; // [batch] index of the sequence's block 0 in kb_tok0 / kb_ntok / kb_dst
   const int64_t* seq_m_off;    // [batch] offset of the sequence inside one head of M ((N_blk - r0) x N_blk entries)
   const int64_t* seq_mt_off;   // [batch] offset of the sequence inside one head of the bit-plane metric
   const int32_t* kb_tok0;      // [n_kb_all] first packed K / V token of every key block (sequence-major)
@@ -65,6 +66,8 @@ struct Plan {
   int32_t k_max = 0, max_nblk = 0;
   int32_t kcache_blocks = 0;  // per-sequence capacity of a caller-owned pooled-K cache (0: none)
   bool share_group = false;   // one index list per (kv head, row)
+  int32_t score_mode = 0;     // 0: product of block means (Eq. 7 on pooled blocks); 1: anti-diagonal scoring
+  std::vector<int32_t> h_seq_r0, h_seq_qtok0;  // host copies: first chunk row, first packed Q token of every sequence
   int32_t H_list = 0;         // heads of the metric and of the lists: H_q, or H_kv with share_group
   int64_t m_tot = 0;
   int64_t mt_tot = 0;  // words per head of the bit-plane metric: sum_b rows(b) * roundup(N_blk(b), 32)
@@ -107,6 +110,13 @@ cudaError_t launch_pool(const Plan& p, const void* Q, const void* K, const void*
 // kernel's tail).  The caller clears status words 4..7 beforehand.
 cudaError_t launch_metric_gemm(const Plan& p, const void* qsplit, const void* ksplit, const float* mv, float* M,
                                bool as_keys, bool dependent, int32_t* status, cudaStream_t s);
+
+// The metric in the anti-diagonal scoring mode, straight from Q and K (mv from the pooling kernel): one tensor-core
+// contraction over the full blocks plus, where a sequence ends in a partial block, a small kernel for that row.
+// *launched receives the number of kernels enqueued.
+int antidiag_max_sequences();
+cudaError_t launch_antidiag_metric(const Plan& p, const void* Q, const void* K, const float* mv, float* M, bool as_keys,
+                                   int32_t* status, int* launched, cudaStream_t s);
 
 // Selection from a stored metric (layout of stem_score's M), one warp per (head, row).
 int row_select_max_blocks();  // largest supported N_blk of a sequence

@@ -54,7 +54,7 @@ extern "C" int stem_score_static(const stem_plan* plan, const void* Q, const voi
   if (!plan || !Q || !K || !V || !M) return STEM_ERR_INVALID_ARG;
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)M) & 15) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;
-  if (p.kcache_blocks > 0) return STEM_ERR_INVALID_ARG;
+  if (p.kcache_blocks > 0 || p.score_mode != 0) return STEM_ERR_INVALID_ARG;
 
   // Size check first: nothing is touched when the problem does not fit.
   const size_t status_bytes = align256(kStatusWords * sizeof(int32_t));
