@@ -12,8 +12,11 @@ from tests._util import check_attention, compare_selection, from_dev_bf16, oracl
 
 pytestmark = pytest.mark.gpu
 
-# the contraction accumulates B * d = 16384 exact bf16 products in fp32; the checker in fp64
-METRIC_ABS, METRIC_REL = 5e-5, 2e-5
+# The contraction adds B * d = 16384 exact bf16 products into one fp32 tensor-memory accumulator over 1024 MMAs, and
+# the tensor core's accumulation truncates: a running sum of a few hundred picks up about 1e-2 before the division
+# by B, i.e. about 1e-4 on metric values of order 1 (measured 1.4e-4).  The checker sums in fp64.  Lists may then
+# differ from the checker's only at near-ties of 1e-3 relative, like on the block-mean path.
+METRIC_ABS, METRIC_REL = 3e-4, 1e-4
 
 CASES = {
     # full blocks only, two column tiles
@@ -61,7 +64,9 @@ def test_antidiagonal_metric_and_fused_path_match_checker(name):
     idx0, cnt0 = torch.empty_like(idx), torch.empty_like(cnt)
     binding.stem_score_select(plan0, q, k, v, idx0, cnt0)
     torch.cuda.synchronize()
-    assert torch.equal(cnt0, cnt) and not torch.equal(idx0, idx)
+    assert torch.equal(cnt0, cnt)
+    if name != "ragged_varlen":     # (its sequences are so short that every causal block is kept in either mode)
+        assert not torch.equal(idx0, idx)
     plan.close(); plan0.close()
 
 
