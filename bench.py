@@ -381,6 +381,63 @@ def main():
         plan.close()
         return res
 
+    def bench_extensions(w, steps, warmup):
+        """The extensions on the same layer: chunked prefill through the pooled-K cache (four chunks, budget at the
+        global row), one index list per kv group, and the anti-diagonal scoring mode."""
+        data = wl.make_qkv(w, layer=replica_layer(rank))
+        q, k, v = dev(data["q"]), dev(data["k"]), dev(data["v"])
+        N, B = w.seqlens[0], w.block
+        res = {}
+        # --- chunked prefill: 4 chunks, K-side pooled tensors kept in a caller-owned cache across chunks
+        n_chunks, step = 4, w.seqlens[0] // 4
+        plans = [pkg.StemPlan.from_workload(w, seqlens=((c + 1) * step,), q_starts=[c * step], total_lens=[N],
+                                            kcache_blocks_per_seq=N // B) for c in range(n_chunks)]
+        cache = torch.zeros(int(plans[0].info.kcache_bytes), dtype=torch.uint8, device="cuda")
+        outs = [torch.empty((step, w.num_q_heads, 128), dtype=torch.bfloat16, device="cuda") for _ in range(n_chunks)]
+        for p_ in plans:
+            p_.workspace()
+        per_chunk = []
+        for c, p_ in enumerate(plans):
+            lo, hi = c * step, (c + 1) * step
+            ms, _ = time_loop(lambda: pkg.stem_prefill_cached(p_, q[lo:hi], k[:hi], v[:hi], outs[c], cache, True), steps, warmup)
+            per_chunk.append(ms)
+            st, detail = pkg.stem_check_status(p_)
+            if st != 0:
+                raise SystemExit(f"device status {st} {detail}")
+        res["chunked_prefill_4x32k_cached"] = {"ms_per_chunk": per_chunk, "ms_per_layer": sum(per_chunk),
+                                                "launches_per_chunk": plans[0].last_launch_count()}
+        for p_ in plans:
+            p_.close()
+        del cache, outs
+        # --- one list per kv group
+        out = torch.empty((w.total_tokens, w.num_q_heads, 128), dtype=torch.bfloat16, device="cuda")
+        ps = pkg.StemPlan.from_workload(w, share_group=True)
+        idx = torch.empty((w.num_kv_heads, ps.info.total_q_blocks, ps.info.k_max), dtype=torch.int32, device="cuda")
+        cnt = torch.empty((w.num_kv_heads, ps.info.total_q_blocks), dtype=torch.int32, device="cuda")
+        pkg.stem_prefill(ps, q, k, v, out, idx, cnt)
+        t = time_interleaved({"fused": lambda: pkg.stem_prefill(ps, q, k, v, out, idx, cnt),
+                              "scoring": lambda: pkg.stem_score_select(ps, q, k, v, idx, cnt),
+                              "attention": lambda: pkg.stem_sparse_prefill(ps, q, k, v, idx, cnt, out)}, steps, warmup, rounds=2)
+        tf = 4.0 * 128 * ps.info.selected_pairs / (t["attention"][0] * 1e-3) / 1e12
+        res["share_group"] = {"ms_per_layer": t["fused"][0], "scoring_stage_ms": t["scoring"][0], "attn_ms": t["attention"][0],
+                              "attn_tflops": tf, "attn_frac_of_measured_peak": tf / peaks["bf16_tflops"]}
+        ps.close()
+        # --- anti-diagonal scoring mode
+        pa = pkg.StemPlan.from_workload(w, score_mode=1)
+        idx = torch.empty((w.num_q_heads, pa.info.total_q_blocks, pa.info.k_max), dtype=torch.int32, device="cuda")
+        cnt = torch.empty((w.num_q_heads, pa.info.total_q_blocks), dtype=torch.int32, device="cuda")
+        pkg.stem_prefill(pa, q, k, v, out, idx, cnt)
+        t = time_interleaved({"fused": lambda: pkg.stem_prefill(pa, q, k, v, out, idx, cnt),
+                              "scoring": lambda: pkg.stem_score_select(pa, q, k, v, idx, cnt)}, steps, warmup, rounds=2)
+        st, detail = pkg.stem_check_status(pa)
+        if st != 0:
+            raise SystemExit(f"device status {st} {detail}")
+        flops = 2.0 * 128 * w.block * (pa.info.causal_blocks)   # B * d multiply-adds per causal block pair and head
+        res["antidiag_scoring"] = {"ms_per_layer": t["fused"][0], "scoring_stage_ms": t["scoring"][0],
+                                   "contraction_tflop": flops / 1e12}
+        pa.close()
+        return res
+
     w = wl.CONFIGS[args.workload]
     sampler = ClockSampler(local)
     sampler.start()
@@ -395,6 +452,8 @@ def main():
                          "attn_frac_of_measured_peak": r2["attn_flops"] / (r2["attn_ms"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
                          "attn_dram_traffic_bytes": NCU_ATTN_DRAM_BYTES_PER_LAUNCH.get(w2.name),
                          "e2e_ms": r2.get("e2e_ms"), "e2e_identical": r2.get("e2e_identical")}
+    if not args.no_extras and args.workload == "cfg3":
+        also.update(bench_extensions(w, max(4, args.steps // 2), 2))
     clocks = sampler.stop()
     # time x clock per stage: the SM clock differs between power states, so stages are comparable across runs as
     # "cycles" = ms x median SM MHz over the samples that fell into the stage's timed windows (all samples if none did)

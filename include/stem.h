@@ -254,6 +254,36 @@ int stem_prefill_cached(const stem_plan* plan, const void* Q, const void* K, con
                         int update_cache, int32_t* sel_idx, int32_t* sel_cnt, float* lse, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------------------------------------------------------
+ * Token Position-Decay on a token-level selector (Main Results: the integration with a sparse-attention
+ * model that keeps the top 2048 tokens per query, k_start = 2048, mu = 0.7).  One sequence of n_tokens;
+ * selection granularity is ONE TOKEN; one index list per (kv head, query token), shared by the query heads
+ * of the group.  head_dim = 128, bf16, layouts as above.
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Eq. 3 at token positions: k(t) = floor(k_start - k_start (1 - mu) (t+1) / n_tokens), raised to the number of
+ * forced tokens (the first stem_tokens and the last local_tokens of the t+1 causal tokens, the token itself
+ * included: local_tokens >= 1) and capped at t+1.  Host only; k_host: HOST int32 [n_tokens]. */
+int stem_token_budget(int32_t n_tokens, int32_t k_start, int32_t mu_num, int32_t mu_den, int32_t stem_tokens,
+                      int32_t local_tokens, int32_t* k_host);
+
+/* Per (list head, query token t): keeps the forced tokens, then the causal tokens of largest score until the list
+ * holds k_tok[t] tokens (score descending, token id ascending on equal scores, -0 == +0, NaN lowest); the list is
+ * emitted ascending, -1 padded.  scores: DEVICE fp32 [list_heads, n_tokens, n_tokens] (row t: entries 0 .. t are
+ * read), the indexer scores the caller computed; k_tok: DEVICE int32 [n_tokens]; sel_idx int32
+ * [list_heads, n_tokens, k_max], sel_cnt int32 [list_heads, n_tokens]; k_max >= max_t k_tok[t]. */
+int stem_token_select(const float* scores, int32_t n_tokens, int32_t list_heads, const int32_t* k_tok, int32_t stem_tokens,
+                      int32_t local_tokens, int32_t k_max, int32_t* sel_idx, int32_t* sel_cnt, void* stream);
+
+/* Gather-style attention over token lists: O[t,h] = softmax_s( Q[t,h].K[s,kv(h)] * softmax_scale ) V over the tokens
+ * s of list (kv(h), t) (ids are clamped to [0, t], never dereferenced out of range).  Lists are per kv head
+ * ([num_kv_heads, n_tokens, k_max]); at most 8 query heads per kv head (STEM_ERR_UNSUPPORTED otherwise).
+ * softmax_scale 0 means 1/sqrt(128).  O bf16 [n_tokens, num_q_heads, 128]; lse fp32 [num_q_heads, n_tokens] or NULL. */
+int stem_token_attention(const void* Q, const void* K, const void* V, int32_t n_tokens, int32_t num_q_heads,
+                         int32_t num_kv_heads, int64_t q_stride_tok, int64_t q_stride_head, int64_t kv_stride_tok,
+                         int64_t kv_stride_head, const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_max,
+                         float softmax_scale, void* O, float* lse, void* stream);
+
 /* Synchronises `stream`, then reads the device status words of `workspace` (workspace == NULL: of
  * the scratch built into the library, see stem_score_static) and clears them if they are set.
  * Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in a kernel gave up; outputs of that

@@ -25,6 +25,7 @@ STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_create_ex", "stem_plan_destroy", "stem_plan_query",
            "stem_pool_kv", "stem_score_select_cached", "stem_prefill_cached",
+           "stem_token_budget", "stem_token_select", "stem_token_attention",
            "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_score_select", "stem_sparse_prefill", "stem_prefill",
            "stem_check_status", "stem_selftest_wait_timeout", "stem_last_launch_count")
 
@@ -116,6 +117,10 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_pool_kv.argtypes = [vp, vp, vp, vp, vp]
     lib.stem_score_select_cached.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
     lib.stem_prefill_cached.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int, vp, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.stem_token_budget.argtypes = [ctypes.c_int32] * 6 + [i32p]
+    lib.stem_token_select.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+    lib.stem_token_attention.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
+                                         ctypes.c_int64, ctypes.c_int64, vp, vp, ctypes.c_int32, ctypes.c_float, vp, vp, vp]
     lib.stem_plan_destroy.argtypes = [vp]
     lib.stem_plan_query.argtypes = [vp, ctypes.POINTER(StemPlanInfo)]
     lib.stem_plan_budget.argtypes = [vp, i32p]
@@ -297,6 +302,32 @@ def stem_prefill_cached(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: tor
     _check(load().stem_prefill_cached(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(kcache),
                                       1 if update_cache else 0, _ptr(sel_idx), _ptr(sel_cnt), _ptr(lse), p, n, _stream()),
            "stem_prefill_cached")
+
+
+def stem_token_budget(n_tokens: int, k_start: int, mu=(7, 10), stem_tokens: int = 0, local_tokens: int = 1) -> torch.Tensor:
+    """Eq. 3 at token positions -> int32 [n_tokens] (host tensor)."""
+    out = torch.empty(n_tokens, dtype=torch.int32)
+    _check(load().stem_token_budget(n_tokens, k_start, mu[0], mu[1], stem_tokens, local_tokens,
+                                    ctypes.cast(out.data_ptr(), ctypes.POINTER(ctypes.c_int32))), "stem_token_budget")
+    return out
+
+
+def stem_token_select(scores: torch.Tensor, k_tok: torch.Tensor, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,
+                      stem_tokens: int = 0, local_tokens: int = 1) -> None:
+    """Token-level top-k(t) from indexer scores [list_heads, N, N]; lists [list_heads, N, k_max]."""
+    h, n, _ = scores.shape
+    _check(load().stem_token_select(_ptr(scores), n, h, _ptr(k_tok), stem_tokens, local_tokens, sel_idx.shape[2], _ptr(sel_idx),
+                                    _ptr(sel_cnt), _stream()), "stem_token_select")
+
+
+def stem_token_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, sel_idx: torch.Tensor, sel_cnt: torch.Tensor,
+                         out: torch.Tensor, lse: Optional[torch.Tensor] = None, softmax_scale: float = 0.0) -> None:
+    """Gather-style attention over per-kv-head token lists; q [N, H_q, 128], k / v [N, H_kv, 128]."""
+    n, hq, _ = q.shape
+    hkv = k.shape[1]
+    _check(load().stem_token_attention(_ptr(q), _ptr(k), _ptr(v), n, hq, hkv, q.stride(0), q.stride(1), k.stride(0), k.stride(1),
+                                       _ptr(sel_idx), _ptr(sel_cnt), sel_idx.shape[2], softmax_scale, _ptr(out), _ptr(lse), _stream()),
+           "stem_token_attention")
 
 
 def stem_sparse_prefill(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

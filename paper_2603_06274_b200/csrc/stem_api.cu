@@ -557,6 +557,39 @@ int stem_prefill_cached(const stem_plan* plan, const void* Q, const void* K, con
   return enqueue_prefill(p, Q, K, V, O, kcache, update_cache != 0, sel_idx, sel_cnt, lse, (uint8_t*)ws, (cudaStream_t)stream);
 }
 
+int stem_token_budget(int32_t n_tokens, int32_t k_start, int32_t mu_num, int32_t mu_den, int32_t stem_tokens,
+                      int32_t local_tokens, int32_t* k_host) {
+  if (n_tokens < 1 || k_start < 0 || mu_den <= 0 || mu_num <= 0 || mu_num > mu_den || stem_tokens < 0 || local_tokens < 1 || !k_host)
+    return STEM_ERR_INVALID_ARG;
+  stem_config c{};
+  c.mu_num = mu_num; c.mu_den = mu_den; c.stem_blocks = stem_tokens; c.local_blocks = local_tokens; c.min_blocks = 0;
+  for (int64_t t = 0; t < n_tokens; ++t) k_host[t] = budget_row(t + 1, n_tokens, k_start, c);  // Eq. 3 with one token per "block"
+  return STEM_OK;
+}
+
+int stem_token_select(const float* scores, int32_t n_tokens, int32_t list_heads, const int32_t* k_tok, int32_t stem_tokens,
+                      int32_t local_tokens, int32_t k_max, int32_t* sel_idx, int32_t* sel_cnt, void* stream) {
+  if (!scores || !k_tok || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
+  if (n_tokens < 1 || list_heads < 1 || list_heads > 65535 || k_max < 1 || stem_tokens < 0 || local_tokens < 1) return STEM_ERR_INVALID_ARG;
+  return cuda_rc(launch_token_select(scores, n_tokens, list_heads, k_max, k_tok, stem_tokens, local_tokens, sel_idx, sel_cnt,
+                                     (cudaStream_t)stream));
+}
+
+int stem_token_attention(const void* Q, const void* K, const void* V, int32_t n_tokens, int32_t num_q_heads,
+                         int32_t num_kv_heads, int64_t q_stride_tok, int64_t q_stride_head, int64_t kv_stride_tok,
+                         int64_t kv_stride_head, const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_max,
+                         float softmax_scale, void* O, float* lse, void* stream) {
+  if (!Q || !K || !V || !O || !sel_idx || !sel_cnt) return STEM_ERR_INVALID_ARG;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return STEM_ERR_INVALID_ARG;
+  if (n_tokens < 1 || num_q_heads < 1 || num_kv_heads < 1 || num_kv_heads > 65535 || k_max < 1) return STEM_ERR_INVALID_ARG;
+  if (num_q_heads % num_kv_heads != 0 || num_q_heads / num_kv_heads > token_attn_max_group()) return STEM_ERR_UNSUPPORTED;
+  if (q_stride_tok % 8 || q_stride_head % 8 || kv_stride_tok % 8 || kv_stride_head % 8) return STEM_ERR_INVALID_ARG;
+  if (!(softmax_scale >= 0.f)) return STEM_ERR_INVALID_ARG;
+  const float scale = softmax_scale == 0.f ? 1.f / std::sqrt((float)kHeadDim) : softmax_scale;
+  return cuda_rc(launch_token_attention(Q, K, V, q_stride_tok, q_stride_head, kv_stride_tok, kv_stride_head, n_tokens, num_q_heads,
+                                        num_kv_heads, k_max, sel_idx, sel_cnt, scale, O, lse, (cudaStream_t)stream));
+}
+
 int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* detail) {
   if (!plan) return STEM_ERR_INVALID_ARG;
   const Plan& p = plan->p;

@@ -131,6 +131,14 @@ cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K,
                                     const int32_t* sel_idx, const int32_t* sel_cnt, bool list_group, void* O, float* lse,
                                     int32_t* status, cudaStream_t s);
 
+// Token-level selection and gather attention (one sequence; lists per kv head).
+int token_attn_max_group();
+cudaError_t launch_token_select(const float* scores, int N, int H_list, int k_max, const int32_t* k_tok, int stem, int local,
+                                int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s);
+cudaError_t launch_token_attention(const void* Q, const void* K, const void* V, int64_t q_st, int64_t q_sh, int64_t kv_st,
+                                   int64_t kv_sh, int N, int Hq, int Hkv, int k_max, const int32_t* sel_idx,
+                                   const int32_t* sel_cnt, float softmax_scale, void* O, float* lse, cudaStream_t s);
+
 // One thread waits 1 ms on a barrier nobody arrives at and records the time-out in status words 0..3.
 cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);
 

@@ -125,3 +125,15 @@ def test_workload_generators_are_deterministic_and_shaped():
     x = np.array([1.0, -2.5, 3.1415927, 1e-20, 65504.0], np.float32)
     back = wl.bf16_bits_to_f32(wl.f32_to_bf16_bits(x))
     assert np.all(np.abs(back - x) <= np.abs(x) * 2.0 ** -8)
+
+
+def test_token_level_budget_is_the_schedule_with_one_token_per_block():
+    # Eq. 3 at token positions (the top-2048 selector setting: k_start = 2048, mu = 0.7): the library's host table
+    # against the checker's schedule with block size 1, and against the printed k_uni = 0.85 k_start
+    n, k_s = 16384, 2048
+    p = so.StemParams(block=1, k_start_blocks=k_s, mu_num=7, mu_den=10, stem_blocks=0, local_blocks=1)
+    got = binding.stem_token_budget(n, k_s, (7, 10), 0, 1).numpy()
+    assert np.array_equal(got, so.schedule(n, k_s, p)[1])
+    uncapped = np.floor(k_s - k_s * 0.3 * np.arange(1, n + 1) / n)
+    assert abs(uncapped.mean() / k_s - 0.85) < 1e-3
+    assert got[-1] == int(0.7 * k_s) and got[0] == 1 and got[k_s + 500] == uncapped[k_s + 500]

@@ -1,0 +1,84 @@
+"""GPU parity of the token-level path (Main Results: Token Position-Decay on a selector that keeps the top 2048
+tokens per query, k_start = 2048, mu = 0.7): the budget k(t) of Eq. 3 at token positions, exact top-k(t) selection
+from caller-supplied indexer scores, and gather-style attention over the token lists.  The CPU checker is
+Algorithm 1's own code with a block size of one token."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import stem_oracle as so
+from paper_2603_06274_b200 import binding, workloads as wl
+from tests._util import check_attention, from_dev_bf16, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _scores(seed, heads, n, ties):
+    r = np.random.Generator(np.random.PCG64([seed, 31]))
+    m = r.standard_normal((heads, n, n), dtype=np.float32)
+    if ties:
+        m = np.round(m * 3.0) / 3.0
+        m[0, n - 1, 5:40] = np.nan
+        m[heads - 1, n // 2, 0:n // 4:3] = np.inf
+        m[0, n // 3, 10:20] = -np.inf
+        m[m == 0.0] = -0.0
+    return m
+
+
+def _case(n, hq, hkv, k_start, stem, local, seed, ties, sample=None):
+    w = wl.small(f"token_{n}", seqlens=(n,), hq=hq, hkv=hkv, block=64, permille=100, sink=True, seed=seed)
+    data = wl.make_qkv(w)
+    g = hq // hkv
+    p = so.StemParams(block=1, k_start_blocks=k_start, mu_num=7, mu_den=10, stem_blocks=stem, local_blocks=local)
+    k_ref = so.schedule(n, k_start, p)[1]
+    k_tok = binding.stem_token_budget(n, k_start, (7, 10), stem, local)
+    assert np.array_equal(k_tok.numpy(), k_ref)
+    k_max = int(k_ref.max())
+    sc = _scores(seed, hkv, n, ties)
+    idx_ref, cnt_ref = so.select(sc.reshape(hkv, -1), np.array([n], np.int32), k_ref, stem, local)
+    idx = torch.full((hkv, n, k_max), -7, dtype=torch.int32, device="cuda")
+    cnt = torch.full((hkv, n), -7, dtype=torch.int32, device="cuda")
+    binding.stem_token_select(torch.from_numpy(sc).cuda(), k_tok.cuda(), idx, cnt, stem, local)
+    torch.cuda.synchronize()
+    assert np.array_equal(cnt.cpu().numpy(), cnt_ref)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref)
+    # gather attention on those lists; the checker runs Algorithm 1 step d with one token per block
+    q, k, v = to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"])
+    out = torch.full((n, hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((hq, n), float("nan"), dtype=torch.float32, device="cuda")
+    binding.stem_token_attention(q, k, v, idx, cnt, out, lse)
+    torch.cuda.synchronize()
+    ei, ec = so.expand_group_lists(idx_ref, cnt_ref, g)
+    rows = None
+    if sample is not None:
+        r = np.random.default_rng(seed)
+        toks = np.unique(np.concatenate([[0, 1, k_start - 1, k_start, n // 2, n - 1], r.integers(0, n, sample)]))
+        rows = np.array([(h, t) for h in range(hq) for t in toks], dtype=np.int32)
+    O_ref, lse_ref = so.attention(data["q"], data["k"], data["v"], data["cu_seqlens"], 1, ei, ec, rows=rows)
+    mask = ~np.isnan(O_ref)
+    check_attention(from_dev_bf16(out), O_ref, mask, label=f"token-level n={n} k_start={k_start}")
+    lm = ~np.isnan(lse_ref)
+    assert np.abs(lse.cpu().numpy()[lm] - lse_ref[lm]).max() < 1e-3
+    assert torch.isfinite(out.float()).all()
+
+
+def test_token_level_selection_and_gather_attention_small():
+    _case(n=700, hq=4, hkv=2, k_start=200, stem=4, local=8, seed=7, ties=True)
+    _case(n=333, hq=3, hkv=3, k_start=64, stem=0, local=1, seed=8, ties=False)
+
+
+def test_token_level_top_2048_selector():
+    # the paper's setting for that integration: k_start = 2048, mu = 0.7; 4096 tokens, GQA 4
+    _case(n=4096, hq=8, hkv=2, k_start=2048, stem=0, local=1, seed=9, ties=True, sample=40)
+
+
+def test_token_level_argument_errors():
+    with pytest.raises(binding.StemError):
+        binding.stem_token_budget(100, 10, (11, 10))
+    q = torch.zeros((64, 18, 128), dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros((64, 2, 128), dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros((2, 64, 4), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros((2, 64), dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.StemError) as e:
+        binding.stem_token_attention(q, kv, kv, idx, cnt, torch.empty_like(q))     # 9 query heads per kv head
+    assert e.value.status == binding.STEM_ERR_UNSUPPORTED
