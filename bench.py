@@ -436,6 +436,29 @@ def main():
         res["antidiag_scoring"] = {"ms_per_layer": t["fused"][0], "scoring_stage_ms": t["scoring"][0],
                                    "contraction_tflop": flops / 1e12}
         pa.close()
+        del q, k, v, out, idx, cnt
+        # --- token-level selector (k_start = 2048, mu = 0.7) on the same head layout at 8K tokens
+        wt = w.with_(seqlens=(8192,), name="token_level_8k")
+        dt = wl.make_qkv(wt, layer=replica_layer(rank))
+        q, k, v = dev(dt["q"]), dev(dt["k"]), dev(dt["v"])
+        n, hkv = 8192, wt.num_kv_heads
+        k_tok = pkg.stem_token_budget(n, 2048, (7, 10), 0, 1)
+        k_max = int(k_tok.max())
+        gen = torch.Generator(device="cuda"); gen.manual_seed(wt.seed)
+        scores = torch.randn((hkv, n, n), dtype=torch.float32, device="cuda", generator=gen)   # stands in for an indexer's output
+        idx = torch.empty((hkv, n, k_max), dtype=torch.int32, device="cuda")
+        cnt = torch.empty((hkv, n), dtype=torch.int32, device="cuda")
+        out = torch.empty((n, wt.num_q_heads, 128), dtype=torch.bfloat16, device="cuda")
+        k_dev = k_tok.cuda()
+        t = time_interleaved({"select": lambda: pkg.stem_token_select(scores, k_dev, idx, cnt, 0, 1),
+                              "attention": lambda: pkg.stem_token_attention(q, k, v, idx, cnt, out)}, steps, warmup, rounds=2)
+        listed = int(k_tok.sum()) * hkv
+        score_bytes = hkv * n * (n + 1) // 2 * 4
+        res["token_level_top2048_8k"] = {"select_ms": t["select"][0], "attention_ms": t["attention"][0],
+                                         "select_gbs_on_causal_scores": score_bytes / (t["select"][0] * 1e-3) / 1e9,
+                                         "gathered_gb_per_launch": listed * 512 / 1e9,
+                                         "gather_gbs": listed * 512 / (t["attention"][0] * 1e-3) / 1e9,
+                                         "attention_tflops": 4.0 * 128 * listed * (wt.num_q_heads // hkv) / (t["attention"][0] * 1e-3) / 1e12}
         return res
 
     w = wl.CONFIGS[args.workload]

@@ -8,8 +8,8 @@
 //                         (score descending, token id ascending) with a four-pass radix selection on
 //                         order-preserving keys through shared-memory histograms; the forced tokens (the first
 //                         `stem` and the last `local`, the token itself included) are kept outside the
-//                         ranking; the list comes out ascending.  Reads the score row from memory twice
-//                         (a row is at most 128 KB and stays in the L2).
+//                         ranking; the list comes out ascending.  The row's keys are converted once into
+//                         shared memory (rows of up to 51 200 tokens; longer rows are re-read from the L2).
 //   token_attn_kernel     gather-style attention: one CTA per (query token, kv head) walks the token list;
 //                         the g query heads of the group share every gathered K / V row.  Scores with one
 //                         key per lane (a lane reads its key's whole row), probabilities times values with one
@@ -60,15 +60,20 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* 
   return base + incl - v;
 }
 
+// kInSmem: the row's candidate keys are converted once and kept in (dynamic) shared memory, so the score row is
+// read from memory a single time; rows too long for that are re-read from memory (they stay in the L2).
+template <bool kInSmem>
 __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* __restrict__ scores, int N, int k_max,
                                                                    const int32_t* __restrict__ k_tok, int stem, int local,
                                                                    int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
-  __shared__ int hist[256];
+  extern __shared__ uint32_t s_keys[];
+  __shared__ int hist[kSelThreads / 32][256];  // one histogram per warp: fewer colliding atomics
   __shared__ int warp_sums[kSelThreads / 32];
   __shared__ uint32_t s_prefix;
   __shared__ int s_need;
   const int t = N - 1 - (int)blockIdx.x;  // long rows first
   const int lh = blockIdx.y;
+  const int warp = threadIdx.x >> 5;
   const int i = t + 1;                                                    // causal tokens 0 .. t
   const int n_stem = min(stem, i);
   const int c_lo = n_stem, c_hi = max(max(i - local, 0), n_stem);         // candidates [c_lo, c_hi)
@@ -77,29 +82,59 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
   const int need = max(min(k_tok[t] - n_forced, n_cand), 0);
   const float* row = scores + ((int64_t)lh * N + t) * N;
   int32_t* out = sel_idx + ((int64_t)lh * N + t) * k_max;
+  auto key_at = [&](int c) -> uint32_t { return kInSmem ? s_keys[c - c_lo] : score_key(row[c]); };
 
+  const bool ranked = need > 0 && need < n_cand;  // otherwise none or all of the candidates are taken
+  if (kInSmem && ranked) {
+    for (int c = c_lo + (int)threadIdx.x; c < c_hi; c += kSelThreads) s_keys[c - c_lo] = score_key(row[c]);
+    __syncthreads();
+  }
   // ---- the need-th largest key: most significant byte first, a histogram per byte
   uint32_t prefix = 0u;  // the bytes decided so far (in the high bits)
   int k = need;          // rank wanted among the keys that match the prefix
-  if (need > 0 && need < n_cand) {
+  if (ranked) {
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-      hist[threadIdx.x] = 0;
+#pragma unroll
+      for (int w = 0; w < kSelThreads / 32; ++w) hist[w][threadIdx.x] = 0;
       __syncthreads();
       for (int c = c_lo + (int)threadIdx.x; c < c_hi; c += kSelThreads) {
-        const uint32_t key = score_key(row[c]);
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+        const uint32_t key = key_at(c);
+        if ((key & mask) == prefix) atomicAdd(&hist[warp][(key >> shift) & 255u], 1);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        int acc = 0, b = 255;
-        for (; b > 0; --b) {  // largest byte value whose count reaches the rank
-          if (acc + hist[b] >= k) break;
-          acc += hist[b];
+      {
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < kSelThreads / 32; ++w) tot += hist[w][threadIdx.x];
+        __syncthreads();
+        hist[0][threadIdx.x] = tot;
+      }
+      __syncthreads();
+      if (warp == 0) {
+        // the largest byte value b with (number of keys whose byte is >= b) >= k: lane l owns the bins 8 l .. 8 l + 7
+        const int lane = threadIdx.x & 31;
+        int mine = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) mine += hist[0][8 * lane + q];
+        int above = mine;  // keys in the bins of this lane and of the lanes above it
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int u = __shfl_down_sync(0xffffffffu, above, d);
+          if (lane + d < 32) above += u;
         }
-        s_prefix = prefix | ((uint32_t)b << shift);
-        s_need = k - acc;
+        const uint32_t reach = __ballot_sync(0xffffffffu, above >= k);  // lanes at or below the one that holds the rank
+        const int owner = 31 - __clz((int)reach);                        // reach != 0: lane 0 counts every key
+        if (lane == owner) {
+          int acc = above - mine, b = 8 * lane + 7;
+          for (; b > 8 * lane; --b) {
+            if (acc + hist[0][b] >= k) break;
+            acc += hist[0][b];
+          }
+          s_prefix = prefix | ((uint32_t)b << shift);
+          s_need = k - acc;
+        }
       }
       __syncthreads();
       prefix = s_prefix;
@@ -107,20 +142,21 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
       __syncthreads();
     }
   }
-  // keys above `prefix` are taken, of the keys equal to it the first k by token id; need == n_cand takes all
-  const bool take_all = need >= n_cand;
+  // keys above `prefix` are taken, of the keys equal to it the first k by token id
 
   // ---- emission in ascending token order: stem tokens, selected candidates, local tokens
   for (int j = threadIdx.x; j < n_stem; j += kSelThreads) out[j] = j;
   int written = n_stem, eq_seen = 0;
-  if (need > 0) {
+  if (need > 0 && !ranked) {
+    for (int c = c_lo + (int)threadIdx.x; c < c_hi; c += kSelThreads) out[n_stem + (c - c_lo)] = c;
+    written += n_cand;
+  } else if (ranked) {
     for (int c0 = c_lo; c0 < c_hi; c0 += kSelThreads) {
       const int c = c0 + (int)threadIdx.x;
-      uint32_t key = 0u;
-      bool in = c < c_hi;
-      if (in) key = score_key(row[c]);
-      const bool gt = in && (take_all || key > prefix);
-      const bool eq = in && !take_all && key == prefix;
+      const bool in = c < c_hi;
+      const uint32_t key = in ? key_at(c) : 0u;
+      const bool gt = in && key > prefix;
+      const bool eq = in && key == prefix;
       int eq_total, sel_total;
       const int eq_before = block_exclusive_scan(eq ? 1 : 0, warp_sums, &eq_total);
       const bool sel = gt || (eq && eq_seen + eq_before < k);
@@ -262,7 +298,23 @@ int token_attn_max_group() { return kMaxGroup; }
 
 cudaError_t launch_token_select(const float* scores, int N, int H_list, int k_max, const int32_t* k_tok, int stem, int local,
                                 int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
-  token_select_kernel<<<dim3((unsigned)N, (unsigned)H_list), kSelThreads, 0, s>>>(scores, N, k_max, k_tok, stem, local, sel_idx, sel_cnt);
+  const dim3 grid((unsigned)N, (unsigned)H_list);
+  const size_t row_bytes = (size_t)N * sizeof(uint32_t);
+  constexpr size_t kSmemLimit = 200 * 1024;
+  if (row_bytes <= kSmemLimit) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!attr_set[dev & 63]) {
+      e = cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+      if (e != cudaSuccess) return e;
+      attr_set[dev & 63] = true;
+    }
+    token_select_kernel<true><<<grid, kSelThreads, row_bytes, s>>>(scores, N, k_max, k_tok, stem, local, sel_idx, sel_cnt);
+  } else {
+    token_select_kernel<false><<<grid, kSelThreads, 0, s>>>(scores, N, k_max, k_tok, stem, local, sel_idx, sel_cnt);
+  }
   return cudaGetLastError();
 }
 
