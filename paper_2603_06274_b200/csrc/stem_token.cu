@@ -37,27 +37,11 @@ __device__ __forceinline__ uint32_t score_key(float f) {
 
 constexpr int kSelThreads = 256;
 
-// Exclusive prefix sum of one value per thread over the CTA (256 threads); *total receives the sum.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int incl = v;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) {
-    const int u = __shfl_up_sync(0xffffffffu, incl, d);
-    if (lane >= d) incl += u;
-  }
-  __syncthreads();  // warp_sums may still be read from the previous call
-  if (lane == 31) warp_sums[warp] = incl;
-  __syncthreads();
-  int base = 0, tot = 0;
-#pragma unroll
-  for (int w = 0; w < kSelThreads / 32; ++w) {
-    const int s = warp_sums[w];
-    if (w < warp) base += s;
-    tot += s;
-  }
-  *total = tot;
-  return base + incl - v;
+// Number of keys equal to the threshold in the segments of the warps before warp w.
+__device__ __forceinline__ int eq_before_all(const int* seg_eq, int w) {
+  int n = 0;
+  for (int q = 0; q < w; ++q) n += seg_eq[q];
+  return n;
 }
 
 // kInSmem: the row's candidate keys are converted once and kept in (dynamic) shared memory, so the score row is
@@ -68,7 +52,6 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
                                                                    int32_t* __restrict__ sel_idx, int32_t* __restrict__ sel_cnt) {
   extern __shared__ uint32_t s_keys[];
   __shared__ int hist[kSelThreads / 32][256];  // one histogram per warp: fewer colliding atomics
-  __shared__ int warp_sums[kSelThreads / 32];
   __shared__ uint32_t s_prefix;
   __shared__ int s_need;
   const int t = N - 1 - (int)blockIdx.x;  // long rows first
@@ -146,25 +129,48 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
 
   // ---- emission in ascending token order: stem tokens, selected candidates, local tokens
   for (int j = threadIdx.x; j < n_stem; j += kSelThreads) out[j] = j;
-  int written = n_stem, eq_seen = 0;
+  int written = n_stem;
   if (need > 0 && !ranked) {
     for (int c = c_lo + (int)threadIdx.x; c < c_hi; c += kSelThreads) out[n_stem + (c - c_lo)] = c;
     written += n_cand;
   } else if (ranked) {
-    for (int c0 = c_lo; c0 < c_hi; c0 += kSelThreads) {
-      const int c = c0 + (int)threadIdx.x;
-      const bool in = c < c_hi;
-      const uint32_t key = in ? key_at(c) : 0u;
-      const bool gt = in && key > prefix;
-      const bool eq = in && key == prefix;
-      int eq_total, sel_total;
-      const int eq_before = block_exclusive_scan(eq ? 1 : 0, warp_sums, &eq_total);
-      const bool sel = gt || (eq && eq_seen + eq_before < k);
-      const int pos = block_exclusive_scan(sel ? 1 : 0, warp_sums, &sel_total);
-      if (sel) out[written + pos] = c;
-      written += sel_total;
-      eq_seen += eq_total;
+    // every warp owns one contiguous segment of the candidates: it counts its keys above and equal to the
+    // threshold, the counts of the warps before it give its first output position, and it then writes its
+    // selected tokens in order (ballots and popcounts, no block-wide step inside the loops)
+    const int lane = threadIdx.x & 31;
+    const int seg = ((n_cand + kSelThreads / 32 - 1) / (kSelThreads / 32) + 31) & ~31;
+    const int s_lo = c_lo + warp * seg, s_hi = min(s_lo + seg, c_hi);
+    int n_gt = 0, n_eq = 0;
+    for (int c0 = s_lo; c0 < s_hi; c0 += 32) {
+      const int c = c0 + lane;
+      const uint32_t key = c < s_hi ? key_at(c) : 0u;
+      n_gt += __popc(__ballot_sync(0xffffffffu, c < s_hi && key > prefix));
+      n_eq += __popc(__ballot_sync(0xffffffffu, c < s_hi && key == prefix));
     }
+    __shared__ int seg_gt[kSelThreads / 32], seg_eq[kSelThreads / 32];
+    if (lane == 0) { seg_gt[warp] = n_gt; seg_eq[warp] = n_eq; }
+    __syncthreads();
+    int eq_before = 0, pos = n_stem, all_sel = 0;
+#pragma unroll
+    for (int w = 0; w < kSelThreads / 32; ++w) {
+      const int take = seg_gt[w] + min(max(k - eq_before_all(seg_eq, w), 0), seg_eq[w]);
+      if (w < warp) { pos += take; eq_before += seg_eq[w]; }
+      all_sel += take;
+    }
+    const uint32_t below = (1u << lane) - 1u;
+    for (int c0 = s_lo; c0 < s_hi; c0 += 32) {
+      const int c = c0 + lane;
+      const uint32_t key = c < s_hi ? key_at(c) : 0u;
+      const bool gt = c < s_hi && key > prefix;
+      const bool eq = c < s_hi && key == prefix;
+      const uint32_t eq_mask = __ballot_sync(0xffffffffu, eq);
+      const bool sel = gt || (eq && eq_before + __popc(eq_mask & below) < k);
+      const uint32_t sel_mask = __ballot_sync(0xffffffffu, sel);
+      if (sel) out[pos + __popc(sel_mask & below)] = c;
+      pos += __popc(sel_mask);
+      eq_before += __popc(eq_mask);
+    }
+    written += all_sel;
   }
   for (int j = c_hi + (int)threadIdx.x; j < i; j += kSelThreads) out[written + (j - c_hi)] = j;
   const int total = written + (i - c_hi);
