@@ -1,5 +1,5 @@
 // One-instruction PTX wrappers and small device helpers shared by the sm_100a kernels of libstem:
-// mbarriers, TMA tile loads, tcgen05 (MMA, commit, fences, tensor-memory loads and stores), the
+// mbarriers, TMA tile loads, tcgen05 (MMA, commit, fences, tensor-memory loads), the
 // shared-memory matrix descriptor, warp election, the global timer, a 32 x 32 bit transpose, and the
 // host-side lookup of the tensor-map encoder.
 #pragma once
@@ -46,40 +46,6 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return done;
 }
-// Non-blocking probe (polling loops over several barriers use this form).
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(done)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return done;
-}
-// Up to four independent probes issued back to back (so their shared-memory round trips overlap);
-// a disabled probe (en == 0) counts as complete.  Returns 1 when every enabled barrier phase is done.
-__device__ __forceinline__ uint32_t mbar_try4(uint32_t b0, uint32_t p0, uint32_t e0, uint32_t b1, uint32_t p1, uint32_t e1,
-                                              uint32_t b2, uint32_t p2, uint32_t e2, uint32_t b3, uint32_t p3, uint32_t e3) {
-  uint32_t done;
-  asm volatile(
-      "{\n\t.reg .pred q0, q1, q2, q3, r0, r1, r2, r3;\n\t"
-      "setp.ne.b32 q0, %3, 0;\n\tsetp.ne.b32 q1, %6, 0;\n\tsetp.ne.b32 q2, %9, 0;\n\tsetp.ne.b32 q3, %12, 0;\n\t"
-      "setp.eq.b32 r0, 0, 0;\n\tsetp.eq.b32 r1, 0, 0;\n\tsetp.eq.b32 r2, 0, 0;\n\tsetp.eq.b32 r3, 0, 0;\n\t"
-      "@q0 mbarrier.try_wait.parity.shared::cta.b64 r0, [%1], %2;\n\t"
-      "@q1 mbarrier.try_wait.parity.shared::cta.b64 r1, [%4], %5;\n\t"
-      "@q2 mbarrier.try_wait.parity.shared::cta.b64 r2, [%7], %8;\n\t"
-      "@q3 mbarrier.try_wait.parity.shared::cta.b64 r3, [%10], %11;\n\t"
-      "and.pred r0, r0, r1;\n\tand.pred r2, r2, r3;\n\tand.pred r0, r0, r2;\n\t"
-      "selp.u32 %0, 1, 0, r0;\n\t}"
-      : "=r"(done)
-      : "r"(b0), "r"(p0), "r"((uint32_t)e0), "r"(b1), "r"(p1), "r"((uint32_t)e1), "r"(b2), "r"(p2), "r"((uint32_t)e2),
-        "r"(b3), "r"(p3), "r"((uint32_t)e3)
-      : "memory");
-  return done;
-}
-
 // Waits for a barrier phase for at most `limit_ns`.  Returns false when the time ran out; the caller
 // records why and unwinds.  `stop` (optional, shared memory) ends the wait early when another role
 // of the CTA has already given up.
@@ -129,15 +95,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
       : "memory");
 }
-// D (tensor memory) (+)= A (tensor memory) x B (shared memory)
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-
 // 32 consecutive 32-bit columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -158,27 +115,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
 // Shared-memory matrix descriptor for tcgen05.mma: 128-byte swizzle, sm_100 descriptor version.
 // K-major operands use lbo = 16, sbo = 1024 (8-row groups 1024 bytes apart).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes = 16, uint32_t sbo_bytes = 1024) {
