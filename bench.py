@@ -196,6 +196,8 @@ def main():
     ap.add_argument("--impl", default="stem", choices=["stem", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the 32K layer, the dense comparator and e2e")
+    ap.add_argument("--e2e-chunks", type=int, default=0,
+                    help="token ranges per kv-head group in the end-to-end pipeline (0: one per 32K tokens, at most 4)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "stem" else args.warmup
     if args.impl == "reference":
@@ -254,10 +256,12 @@ def main():
 
     class GroupPipeline:
         """End-to-end path with host buffers: every kv-head group is independent through all stages, so the groups
-        are pipelined over three streams - H2D of group i+1, Algorithm 1 on group i, D2H of group i-1 - with one
-        strided 2-D copy per tensor slice.  Results are identical to the one-shot call."""
+        are pipelined over three streams - H2D of unit i+1, Algorithm 1 on unit i, D2H of unit i-1 - with one
+        strided 2-D copy per tensor slice.  A single sequence is further cut into `chunks` token ranges per group
+        (chunked prefill: Q holds the range, K / V the prefix up to its end), which shortens the part of the step
+        that no copy can hide: the last unit's kernels and its D2H.  Results are identical to the one-shot call."""
 
-        def __init__(self, w, data):
+        def __init__(self, w, data, chunks=1):
             import ctypes
             self.ct = ctypes
             self.rt = ctypes.CDLL(os.path.join(os.path.dirname(torch.__file__), "lib", "libcudart.so.12")) \
@@ -274,9 +278,17 @@ def main():
             self.v = torch.empty((T, w.num_kv_heads, 128), dtype=torch.bfloat16, device="cuda")
             self.o = [torch.empty((T, self.g, 128), dtype=torch.bfloat16, device="cuda") for _ in range(w.num_kv_heads)]
             # one plan per group: g query heads and one kv head, addressed inside the full tensors by their strides
-            self.plans = [pkg.StemPlan.from_workload(w, num_q_heads=self.g, num_kv_heads=1,
-                                                     q_strides=(w.num_q_heads * 128, 128),
-                                                     kv_strides=(w.num_kv_heads * 128, 128)) for _ in range(w.num_kv_heads)]
+            # (the units run one after another on one stream, so the groups share the plans and their workspaces)
+            strides = dict(num_q_heads=self.g, num_kv_heads=1, q_strides=(w.num_q_heads * 128, 128),
+                           kv_strides=(w.num_kv_heads * 128, 128))
+            if len(w.seqlens) > 1 or chunks <= 1:
+                self.bounds = [0, T]
+                self.plans = [pkg.StemPlan.from_workload(w, **strides)]
+            else:
+                nblk = (T + w.block - 1) // w.block
+                self.bounds = sorted({min(T, (nblk * c // chunks) * w.block) for c in range(chunks)} | {T})
+                self.plans = [pkg.StemPlan.from_workload(w, seqlens=[t1], q_starts=[t0], total_lens=[T], **strides)
+                              for t0, t1 in zip(self.bounds[:-1], self.bounds[1:])]
             for p in self.plans:
                 p.workspace()
             self.s_in, self.s_out = torch.cuda.Stream(), torch.cuda.Stream()
@@ -296,23 +308,28 @@ def main():
             start = torch.cuda.Event(); start.record(cur)
             self.s_in.wait_event(start)
             last_out = None
+            self.launches = 0
             for i in range(w.num_kv_heads):
                 if self.done[i] is not None:
                     self.s_in.wait_event(self.done[i])   # the previous step's kernels may still read this slice
                 qp, kp = w.num_q_heads * 256, w.num_kv_heads * 256
-                self._copy2d(self.q.data_ptr() + i * g * 256, qp, self.hq.data_ptr() + i * g * 256, qp, g * 256, T, 1, self.s_in)
-                self._copy2d(self.k.data_ptr() + i * 256, kp, self.hk.data_ptr() + i * 256, kp, 256, T, 1, self.s_in)
-                self._copy2d(self.v.data_ptr() + i * 256, kp, self.hv.data_ptr() + i * 256, kp, 256, T, 1, self.s_in)
-                arrived = torch.cuda.Event(); arrived.record(self.s_in)
-                cur.wait_event(arrived)
-                pkg.stem_prefill(self.plans[i], self.q[:, i * g:(i + 1) * g], self.k[:, i:i + 1], self.v[:, i:i + 1], self.o[i])
-                computed = torch.cuda.Event(); computed.record(cur)
-                self.done[i] = computed
-                self.s_out.wait_event(computed)
-                self._copy2d(self.ho.data_ptr() + i * g * 256, qp, self.o[i].data_ptr(), g * 256, g * 256, T, 2, self.s_out)
-                last_out = torch.cuda.Event(); last_out.record(self.s_out)
+                for plan, t0, t1 in zip(self.plans, self.bounds[:-1], self.bounds[1:]):
+                    n = t1 - t0
+                    self._copy2d(self.q.data_ptr() + t0 * qp + i * g * 256, qp, self.hq.data_ptr() + t0 * qp + i * g * 256, qp,
+                                 g * 256, n, 1, self.s_in)
+                    self._copy2d(self.k.data_ptr() + t0 * kp + i * 256, kp, self.hk.data_ptr() + t0 * kp + i * 256, kp, 256, n, 1, self.s_in)
+                    self._copy2d(self.v.data_ptr() + t0 * kp + i * 256, kp, self.hv.data_ptr() + t0 * kp + i * 256, kp, 256, n, 1, self.s_in)
+                    arrived = torch.cuda.Event(); arrived.record(self.s_in)
+                    cur.wait_event(arrived)
+                    pkg.stem_prefill(plan, self.q[t0:t1, i * g:(i + 1) * g], self.k[:t1, i:i + 1], self.v[:t1, i:i + 1], self.o[i][t0:t1])
+                    self.launches += plan.last_launch_count()
+                    computed = torch.cuda.Event(); computed.record(cur)
+                    self.done[i] = computed
+                    self.s_out.wait_event(computed)
+                    self._copy2d(self.ho.data_ptr() + t0 * qp + i * g * 256, qp, self.o[i].data_ptr() + t0 * g * 256, g * 256,
+                                 g * 256, n, 2, self.s_out)
+                    last_out = torch.cuda.Event(); last_out.record(self.s_out)
             cur.wait_event(last_out)
-            self.launches = sum(p.last_launch_count() for p in self.plans)
 
         def check(self):
             for p in self.plans:
@@ -369,13 +386,14 @@ def main():
             res["dense_ms"] = time_loop(lambda: pkg.stem_sparse_prefill(plan, q, k, v, None, None, out), dsteps, 1)[0]
             # end to end with HOST buffers: H2D of Q, K, V and D2H of O inside the timed region, every step
             del q, k, v
-            pipe = GroupPipeline(w, data)
+            pipe = GroupPipeline(w, data, chunks=args.e2e_chunks or max(1, min(4, w.total_tokens // 32768)))
             res["e2e_ms"] = time_loop(pipe.step, max(2, min(steps, 5)), 2)[0]
             pipe.check()
             res["e2e_identical"] = bool(torch.equal(torch.cat([o.view(torch.int16) for o in pipe.o], dim=1), fused_out.view(torch.int16))
                                         and torch.equal(pipe.ho.cuda(), fused_out.view(torch.int16)))
             del fused_out
             res["e2e_launches_per_step"] = pipe.launches
+            res["e2e_units"] = w.num_kv_heads * (len(pipe.bounds) - 1)
             res["h2d"], res["d2h"] = int(pipe.h2d), int(pipe.d2h)
             pipe.close()
         plan.close()
@@ -548,8 +566,9 @@ def main():
         "e2e": None if "e2e_ms" not in main_res else {
             "value": main_res["e2e_ms"] / world, "unit": "ms/layer", "h2d_bytes_per_step": main_res["h2d"],
             "d2h_bytes_per_step": main_res["d2h"], "identical_to_one_shot": main_res["e2e_identical"],
-            "launches_per_step": main_res["e2e_launches_per_step"],
-            "how": "kv-head groups pipelined over three streams: H2D of group i+1, Algorithm 1 on group i, D2H of group i-1"},
+            "launches_per_step": main_res["e2e_launches_per_step"], "pipeline_units": main_res["e2e_units"],
+            "how": "units = kv-head groups x token ranges (chunked prefill), pipelined over three streams: H2D of unit i+1, "
+                   "Algorithm 1 on unit i, D2H of unit i-1"},
         "cpu_baseline": cpu,
         "also": also,
     }
