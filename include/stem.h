@@ -276,13 +276,22 @@ int stem_token_select(const float* scores, int32_t n_tokens, int32_t list_heads,
                       int32_t local_tokens, int32_t k_max, int32_t* sel_idx, int32_t* sel_cnt, void* stream);
 
 /* Gather-style attention over token lists: O[t,h] = softmax_s( Q[t,h].K[s,kv(h)] * softmax_scale ) V over the tokens
- * s of list (kv(h), t) (ids are clamped to [0, t], never dereferenced out of range).  Lists are per kv head
- * ([num_kv_heads, n_tokens, k_max]); at most 8 query heads per kv head (STEM_ERR_UNSUPPORTED otherwise).
- * softmax_scale 0 means 1/sqrt(128).  O bf16 [n_tokens, num_q_heads, 128]; lse fp32 [num_q_heads, n_tokens] or NULL. */
+ * s of list (kv(h), t) (ids are clamped to [0, t], never dereferenced out of range; at most min(k_max, t+1) entries
+ * of a list are used).  Lists are per kv head ([num_kv_heads, n_tokens, k_max]); at most 16 query heads per kv head
+ * (STEM_ERR_UNSUPPORTED otherwise).  Strides in elements, multiples of 8; Q, K, V, O 16-byte aligned.
+ * softmax_scale 0 means 1/sqrt(128).  O bf16 [n_tokens, num_q_heads, 128] (contiguous); lse fp32
+ * [num_q_heads, n_tokens] or NULL.  Probabilities are rounded to bf16 before they meet V (as in stem_sparse_prefill).
+ * The call only enqueues; a bounded device-side wait that gave up is reported by stem_token_check_status. */
 int stem_token_attention(const void* Q, const void* K, const void* V, int32_t n_tokens, int32_t num_q_heads,
                          int32_t num_kv_heads, int64_t q_stride_tok, int64_t q_stride_head, int64_t kv_stride_tok,
                          int64_t kv_stride_head, const int32_t* sel_idx, const int32_t* sel_cnt, int32_t k_max,
                          float softmax_scale, void* O, float* lse, void* stream);
+
+/* Synchronises `stream`, then reads (and clears, if set) the status words of the gather-attention kernel on the
+ * current device.  Returns STEM_OK, STEM_ERR_DEVICE_TIMEOUT (a bounded wait in stem_token_attention gave up; the
+ * outputs of that call are undefined) or STEM_ERR_CUDA.  detail (optional, HOST int32[4]) receives
+ * {4, CTA index, role, barrier id}. */
+int stem_token_check_status(void* stream, int32_t* detail_host);
 
 /* Synchronises `stream`, then reads the device status words of `workspace` (workspace == NULL: of
  * the scratch built into the library, see stem_score_static) and clears them if they are set.

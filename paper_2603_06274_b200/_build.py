@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB = os.path.join(_PKG, "libstem.so")
-SOURCES = ["stem_api.cu", "stem_pool.cu", "stem_rowselect.cu", "stem_metric.cu", "stem_antidiag.cu", "stem_attn.cu", "stem_token.cu", "stem_static.cu", "stem_selftest.cu"]
+SOURCES = ["stem_api.cu", "stem_pool.cu", "stem_rowselect.cu", "stem_metric.cu", "stem_antidiag.cu", "stem_attn.cu", "stem_token.cu", "stem_token_attn.cu", "stem_static.cu", "stem_selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

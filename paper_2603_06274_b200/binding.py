@@ -25,7 +25,7 @@ STATIC_SCRATCH_BYTES = 8 * 1024 * 1024
 
 EXPORTS = ("stem_version", "stem_status_string", "stem_plan_create", "stem_plan_create_ex", "stem_plan_destroy", "stem_plan_query",
            "stem_pool_kv", "stem_score_select_cached", "stem_prefill_cached",
-           "stem_token_budget", "stem_token_select", "stem_token_attention",
+           "stem_token_budget", "stem_token_select", "stem_token_attention", "stem_token_check_status",
            "stem_plan_budget", "stem_budget_table", "stem_score", "stem_score_static", "stem_select", "stem_score_select", "stem_sparse_prefill", "stem_prefill",
            "stem_check_status", "stem_selftest_wait_timeout", "stem_last_launch_count")
 
@@ -121,6 +121,7 @@ def load(build_if_missing: bool = True) -> ctypes.CDLL:
     lib.stem_token_select.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
     lib.stem_token_attention.argtypes = [vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64,
                                          ctypes.c_int64, ctypes.c_int64, vp, vp, ctypes.c_int32, ctypes.c_float, vp, vp, vp]
+    lib.stem_token_check_status.argtypes = [vp, i32p]
     lib.stem_plan_destroy.argtypes = [vp]
     lib.stem_plan_query.argtypes = [vp, ctypes.POINTER(StemPlanInfo)]
     lib.stem_plan_budget.argtypes = [vp, i32p]
@@ -328,6 +329,13 @@ def stem_token_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, sel_
     _check(load().stem_token_attention(_ptr(q), _ptr(k), _ptr(v), n, hq, hkv, q.stride(0), q.stride(1), k.stride(0), k.stride(1),
                                        _ptr(sel_idx), _ptr(sel_cnt), sel_idx.shape[2], softmax_scale, _ptr(out), _ptr(lse), _stream()),
            "stem_token_attention")
+
+
+def stem_token_check_status():
+    """Synchronise the current stream and return (status, detail[4]) of the gather-attention kernel."""
+    detail = (ctypes.c_int32 * 4)()
+    st = load().stem_token_check_status(_stream(), ctypes.cast(detail, ctypes.POINTER(ctypes.c_int32)))
+    return int(st), [int(x) for x in detail]
 
 
 def stem_sparse_prefill(plan: StemPlan, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

@@ -584,10 +584,19 @@ int stem_token_attention(const void* Q, const void* K, const void* V, int32_t n_
   if (n_tokens < 1 || num_q_heads < 1 || num_kv_heads < 1 || num_kv_heads > 65535 || k_max < 1) return STEM_ERR_INVALID_ARG;
   if (num_q_heads % num_kv_heads != 0 || num_q_heads / num_kv_heads > token_attn_max_group()) return STEM_ERR_UNSUPPORTED;
   if (q_stride_tok % 8 || q_stride_head % 8 || kv_stride_tok % 8 || kv_stride_head % 8) return STEM_ERR_INVALID_ARG;
+  if (q_stride_head < kHeadDim || kv_stride_head < kHeadDim) return STEM_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.f)) return STEM_ERR_INVALID_ARG;
   const float scale = softmax_scale == 0.f ? 1.f / std::sqrt((float)kHeadDim) : softmax_scale;
   return cuda_rc(launch_token_attention(Q, K, V, q_stride_tok, q_stride_head, kv_stride_tok, kv_stride_head, n_tokens, num_q_heads,
                                         num_kv_heads, k_max, sel_idx, sel_cnt, scale, O, lse, (cudaStream_t)stream));
+}
+
+int stem_token_check_status(void* stream, int32_t* detail) {
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  int32_t words[4] = {0, 0, 0, 0};
+  if (token_status_words(words) != cudaSuccess) { cudaGetLastError(); return STEM_ERR_CUDA; }
+  if (detail) std::memcpy(detail, words, sizeof(words));
+  return words[0] != 0 ? STEM_ERR_DEVICE_TIMEOUT : STEM_OK;
 }
 
 int stem_check_status(const stem_plan* plan, void* ws, void* stream, int32_t* detail) {

@@ -138,6 +138,9 @@ cudaError_t launch_token_select(const float* scores, int N, int H_list, int k_ma
 cudaError_t launch_token_attention(const void* Q, const void* K, const void* V, int64_t q_st, int64_t q_sh, int64_t kv_st,
                                    int64_t kv_sh, int N, int Hq, int Hkv, int k_max, const int32_t* sel_idx,
                                    const int32_t* sel_cnt, float softmax_scale, void* O, float* lse, cudaStream_t s);
+// The status words {4, CTA, role, barrier} of the gather-attention kernel on the current device, read to the host
+// and cleared when set (the caller has synchronised).
+cudaError_t token_status_words(int32_t* out4);
 
 // One thread waits 1 ms on a barrier nobody arrives at and records the time-out in status words 0..3.
 cudaError_t launch_selftest_wait(int32_t* status, cudaStream_t s);

@@ -2,7 +2,7 @@
 // model whose indexer keeps the top 2048 tokens per query; there k_start = 2048 and mu = 0.7).  Selection
 // granularity is one token: query token t keeps k(t) of its t+1 causal tokens, k(t) from Eq. 3 at token
 // positions, ranked by an indexer score the caller supplies (one score matrix per kv head: the heads of a
-// group share the selection), and attends over exactly those tokens.  Two kernels, one sequence:
+// group share the selection), and attends over exactly those tokens.  This file holds the selection:
 //
 //   token_select_kernel   one CTA per (list head, query token): exact top-k of the row's candidates by
 //                         (score descending, token id ascending) with a four-pass radix selection on
@@ -10,14 +10,8 @@
 //                         `stem` and the last `local`, the token itself included) are kept outside the
 //                         ranking; the list comes out ascending.  The row's keys are converted once into
 //                         shared memory (rows of up to 51 200 tokens; longer rows are re-read from the L2).
-//   token_attn_kernel     gather-style attention: one CTA per (query token, kv head) walks the token list;
-//                         the g query heads of the group share every gathered K / V row.  Scores with one
-//                         key per lane (a lane reads its key's whole row), probabilities times values with one
-//                         lane per four output columns (a warp reads a value row coalesced), online softmax
-//                         per warp, the four warps' partial results merged through shared memory.
-//                         Each query token gathers its own rows, so nothing is shared between CTAs except
-//                         through the L2: the kernel is bound by L2 -> SM bandwidth and FMA issue, not by
-//                         the tensor cores (4 g flops per gathered byte).
+//
+// The attention over the lists is in stem_token_attn.cu.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -178,129 +172,7 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
   if (threadIdx.x == 0) sel_cnt[(int64_t)lh * N + t] = total;
 }
 
-// ------------------------------------------------------------------------------------------------
-// gather attention
-// ------------------------------------------------------------------------------------------------
-constexpr int kAttnThreads = 128;
-constexpr int kMaxGroup = 8;  // query heads per kv head
-
-template <int G>
-__global__ void __launch_bounds__(kAttnThreads) token_attn_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
-                                                                  const __nv_bfloat16* __restrict__ V, int64_t q_st, int64_t q_sh,
-                                                                  int64_t kv_st, int64_t kv_sh, int N, int Hq, int k_max,
-                                                                  const int32_t* __restrict__ sel_idx, const int32_t* __restrict__ sel_cnt,
-                                                                  float scale_log2, __nv_bfloat16* __restrict__ O, float* __restrict__ lse) {
-  __shared__ float q_s[G][kHeadDim];          // the group's query vectors, pre-scaled to the log2 domain
-  __shared__ float part_o[4][G][kHeadDim];    // the warps' partial outputs
-  __shared__ float part_m[4][G], part_l[4][G];
-  const int t = N - 1 - (int)blockIdx.x;      // long lists first
-  const int kvh = blockIdx.y;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n = min(max(sel_cnt[(int64_t)kvh * N + t], 0), k_max);
-  const int32_t* list = sel_idx + ((int64_t)kvh * N + t) * k_max;
-
-  for (int e = threadIdx.x; e < G * kHeadDim; e += kAttnThreads) {
-    const int hq = e / kHeadDim, c = e - hq * kHeadDim;
-    q_s[hq][c] = __bfloat162float(Q[(int64_t)t * q_st + (int64_t)(kvh * G + hq) * q_sh + c]) * scale_log2;
-  }
-  __syncthreads();
-
-  float m_run[G], l_run[G], o[G][4];  // per warp: running maxima and sums; this lane's four output columns
-#pragma unroll
-  for (int hq = 0; hq < G; ++hq) {
-    m_run[hq] = -INFINITY;
-    l_run[hq] = 0.f;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) o[hq][c] = 0.f;
-  }
-  const __nv_bfloat16* kbase = K + (int64_t)kvh * kv_sh;
-  const __nv_bfloat16* vbase = V + (int64_t)kvh * kv_sh;
-
-  for (int e0 = warp * 32; e0 < n; e0 += 4 * 32) {
-    // ---- scores: one key per lane
-    const int e = e0 + lane;
-    const bool valid = e < n;
-    const int tok = valid ? min(max(list[e], 0), t) : 0;
-    float s[G];
-#pragma unroll
-    for (int hq = 0; hq < G; ++hq) s[hq] = 0.f;
-    const uint4* krow = (const uint4*)(kbase + (int64_t)tok * kv_st);
-#pragma unroll 4
-    for (int c8 = 0; c8 < kHeadDim / 8; ++c8) {
-      const uint4 kv = krow[c8];
-      const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
-#pragma unroll
-      for (int p = 0; p < 4; ++p) {
-        const float k0 = __uint_as_float(w[p] << 16), k1 = __uint_as_float(w[p] & 0xffff0000u);
-#pragma unroll
-        for (int hq = 0; hq < G; ++hq) s[hq] = fmaf(q_s[hq][c8 * 8 + 2 * p + 1], k1, fmaf(q_s[hq][c8 * 8 + 2 * p], k0, s[hq]));
-      }
-    }
-    // ---- online softmax of the 32 keys, per head
-    float p[G];
-#pragma unroll
-    for (int hq = 0; hq < G; ++hq) {
-      const float sv = valid ? s[hq] : -INFINITY;
-      float mx = sv;
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, d));
-      const float m_new = fmaxf(m_run[hq], mx);
-      const float alpha = exp2f(m_run[hq] - m_new);  // exp2(-inf) = 0 on the first step
-      p[hq] = exp2f(sv - m_new);
-      float ps = p[hq];
-#pragma unroll
-      for (int d = 16; d > 0; d >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, d);
-      l_run[hq] = l_run[hq] * alpha + ps;
-      m_run[hq] = m_new;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) o[hq][c] *= alpha;
-    }
-    // ---- probabilities times values: this lane accumulates columns 4 lane .. 4 lane + 3 of every head
-    const int n_here = min(32, n - e0);
-    for (int j = 0; j < n_here; ++j) {
-      const int tj = __shfl_sync(0xffffffffu, tok, j);
-      const uint2 vv = *(const uint2*)(vbase + (int64_t)tj * kv_st + lane * 4);
-      const float v0 = __uint_as_float(vv.x << 16), v1 = __uint_as_float(vv.x & 0xffff0000u);
-      const float v2 = __uint_as_float(vv.y << 16), v3 = __uint_as_float(vv.y & 0xffff0000u);
-#pragma unroll
-      for (int hq = 0; hq < G; ++hq) {
-        const float pj = __shfl_sync(0xffffffffu, p[hq], j);
-        o[hq][0] = fmaf(pj, v0, o[hq][0]);
-        o[hq][1] = fmaf(pj, v1, o[hq][1]);
-        o[hq][2] = fmaf(pj, v2, o[hq][2]);
-        o[hq][3] = fmaf(pj, v3, o[hq][3]);
-      }
-    }
-  }
-  // ---- merge the four warps
-#pragma unroll
-  for (int hq = 0; hq < G; ++hq) {
-    if (lane == 0) { part_m[warp][hq] = m_run[hq]; part_l[warp][hq] = l_run[hq]; }
-#pragma unroll
-    for (int c = 0; c < 4; ++c) part_o[warp][hq][lane * 4 + c] = o[hq][c];
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < G * kHeadDim; e += kAttnThreads) {
-    const int hq = e / kHeadDim, c = e - hq * kHeadDim;
-    float m = -INFINITY;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) m = fmaxf(m, part_m[w][hq]);
-    float l = 0.f, acc = 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-      const float a = part_m[w][hq] == -INFINITY ? 0.f : exp2f(part_m[w][hq] - m);
-      l += part_l[w][hq] * a;
-      acc += part_o[w][hq][c] * a;
-    }
-    const int h = kvh * G + hq;
-    O[((int64_t)t * Hq + h) * kHeadDim + c] = __float2bfloat16_rn(n > 0 ? acc / l : 0.f);
-    if (lse && c == 0) lse[(int64_t)h * N + t] = n > 0 ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
-  }
-}
-
 }  // namespace
-
-int token_attn_max_group() { return kMaxGroup; }
 
 cudaError_t launch_token_select(const float* scores, int N, int H_list, int k_max, const int32_t* k_tok, int stem, int local,
                                 int32_t* sel_idx, int32_t* sel_cnt, cudaStream_t s) {
@@ -320,28 +192,6 @@ cudaError_t launch_token_select(const float* scores, int N, int H_list, int k_ma
     token_select_kernel<true><<<grid, kSelThreads, row_bytes, s>>>(scores, N, k_max, k_tok, stem, local, sel_idx, sel_cnt);
   } else {
     token_select_kernel<false><<<grid, kSelThreads, 0, s>>>(scores, N, k_max, k_tok, stem, local, sel_idx, sel_cnt);
-  }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_token_attention(const void* Q, const void* K, const void* V, int64_t q_st, int64_t q_sh, int64_t kv_st,
-                                   int64_t kv_sh, int N, int Hq, int Hkv, int k_max, const int32_t* sel_idx,
-                                   const int32_t* sel_cnt, float softmax_scale, void* O, float* lse, cudaStream_t s) {
-  const dim3 grid((unsigned)N, (unsigned)Hkv);
-  const float sl2 = softmax_scale * 1.4426950408889634f;
-  auto q = (const __nv_bfloat16*)Q;
-  auto k = (const __nv_bfloat16*)K;
-  auto v = (const __nv_bfloat16*)V;
-  auto o = (__nv_bfloat16*)O;
-  switch (Hq / Hkv) {
-#define STEM_TOKEN_CASE(G)                                                                                                          \
-  case G:                                                                                                                           \
-    token_attn_kernel<G><<<grid, kAttnThreads, 0, s>>>(q, k, v, q_st, q_sh, kv_st, kv_sh, N, Hq, k_max, sel_idx, sel_cnt, sl2, o, lse); \
-    break;
-    STEM_TOKEN_CASE(1) STEM_TOKEN_CASE(2) STEM_TOKEN_CASE(3) STEM_TOKEN_CASE(4) STEM_TOKEN_CASE(5) STEM_TOKEN_CASE(6) STEM_TOKEN_CASE(7)
-    STEM_TOKEN_CASE(8)
-#undef STEM_TOKEN_CASE
-    default: return cudaErrorInvalidValue;
   }
   return cudaGetLastError();
 }

@@ -47,7 +47,8 @@ def _case(n, hq, hkv, k_start, stem, local, seed, ties, sample=None):
     out = torch.full((n, hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
     lse = torch.full((hq, n), float("nan"), dtype=torch.float32, device="cuda")
     binding.stem_token_attention(q, k, v, idx, cnt, out, lse)
-    torch.cuda.synchronize()
+    st, detail = binding.stem_token_check_status()
+    assert st == 0, detail
     ei, ec = so.expand_group_lists(idx_ref, cnt_ref, g)
     rows = None
     if sample is not None:
@@ -65,6 +66,7 @@ def _case(n, hq, hkv, k_start, stem, local, seed, ties, sample=None):
 def test_token_level_selection_and_gather_attention_small():
     _case(n=700, hq=4, hkv=2, k_start=200, stem=4, local=8, seed=7, ties=True)
     _case(n=333, hq=3, hkv=3, k_start=64, stem=0, local=1, seed=8, ties=False)
+    _case(n=520, hq=8, hkv=1, k_start=300, stem=2, local=3, seed=10, ties=False)   # 8 query heads on one kv head
 
 
 def test_token_level_top_2048_selector():
@@ -75,10 +77,10 @@ def test_token_level_top_2048_selector():
 def test_token_level_argument_errors():
     with pytest.raises(binding.StemError):
         binding.stem_token_budget(100, 10, (11, 10))
-    q = torch.zeros((64, 18, 128), dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((64, 34, 128), dtype=torch.bfloat16, device="cuda")
     kv = torch.zeros((64, 2, 128), dtype=torch.bfloat16, device="cuda")
     idx = torch.zeros((2, 64, 4), dtype=torch.int32, device="cuda")
     cnt = torch.zeros((2, 64), dtype=torch.int32, device="cuda")
     with pytest.raises(binding.StemError) as e:
-        binding.stem_token_attention(q, kv, kv, idx, cnt, torch.empty_like(q))     # 9 query heads per kv head
+        binding.stem_token_attention(q, kv, kv, idx, cnt, torch.empty_like(q))     # 17 query heads per kv head
     assert e.value.status == binding.STEM_ERR_UNSUPPORTED
