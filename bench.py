@@ -470,6 +470,9 @@ def main():
         k_dev = k_tok.cuda()
         t = time_interleaved({"select": lambda: pkg.stem_token_select(scores, k_dev, idx, cnt, 0, 1),
                               "attention": lambda: pkg.stem_token_attention(q, k, v, idx, cnt, out)}, steps, warmup, rounds=2)
+        st, detail = pkg.stem_token_check_status()
+        if st != 0:
+            raise SystemExit(f"device status {st} {detail}")
         listed = int(k_tok.sum()) * hkv
         score_bytes = hkv * n * (n + 1) // 2 * 4
         res["token_level_top2048_8k"] = {"select_ms": t["select"][0], "attention_ms": t["attention"][0],

@@ -176,8 +176,7 @@ antidiag_metric_kernel(const __grid_constant__ MapSet maps, const AntiArgs a) {
 #pragma unroll 1
       for (int gq = 0; gq < 4; ++gq) {
         float v[32];
-        tmem_ld32(taddr + gq * 32, v);
-        tmem_ld_wait();
+        tmem_ld32_sync(taddr + gq * 32, v);
         if (r >= nfull) continue;  // rows of the partial block (or past the end) belong to the other kernel
         if (a.as_keys) {
           uint32_t w[32];

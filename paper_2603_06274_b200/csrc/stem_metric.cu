@@ -197,8 +197,7 @@ metric_gemm_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll 1
       for (int gq = gq0; gq < gq0 + 2; ++gq) {
         float v[32];
-        tmem_ld32(taddr + gq * 32, v);
-        tmem_ld_wait();
+        tmem_ld32_sync(taddr + gq * 32, v);
         if (gq == gq0 + 1) {
           // the accumulator is in registers: the MMAs of head hh + 2 may overwrite it
           tc_fence_before();
