@@ -74,6 +74,11 @@ def test_token_level_top_2048_selector():
     _case(n=4096, hq=8, hkv=2, k_start=2048, stem=0, local=1, seed=9, ties=True, sample=40)
 
 
+def test_token_level_rows_of_9000_tokens():
+    # lists longer than one 2048-token budget window, rows that span several passes of every thread over the keys
+    _case(n=9000, hq=2, hkv=1, k_start=2048, stem=2, local=4, seed=11, ties=True, sample=12)
+
+
 def test_token_level_argument_errors():
     with pytest.raises(binding.StemError):
         binding.stem_token_budget(100, 10, (11, 10))
