@@ -79,6 +79,41 @@ def test_token_level_rows_of_9000_tokens():
     _case(n=9000, hq=2, hkv=1, k_start=2048, stem=2, local=4, seed=11, ties=True, sample=12)
 
 
+def test_gather_attention_on_hand_made_lists_with_strided_tensors():
+    # 16 query heads on one kv head (the widest group), lists of any length from 0 to 140 tokens (a list need not come
+    # from the selector; empty lists give a zero row and lse = -inf), Q / K / V as slices of wider tensors
+    n, hq, hkv = 300, 16, 1
+    w = wl.small("token_lists", seqlens=(n,), hq=hq, hkv=hkv, block=64, permille=100, sink=False, seed=21)
+    data = wl.make_qkv(w)
+    r = np.random.default_rng(21)
+    k_max = 140
+    idx_ref = np.full((hkv, n, k_max), -1, np.int32)
+    cnt_ref = np.zeros((hkv, n), np.int32)
+    for t in range(n):
+        m = 0 if r.random() < 0.1 else int(r.integers(1, min(t + 1, k_max) + 1))
+        idx_ref[0, t, :m] = np.sort(r.choice(t + 1, size=m, replace=False))
+        cnt_ref[0, t] = m
+    q_wide = torch.zeros((n, hq + 4, 128), dtype=torch.bfloat16, device="cuda")
+    k_wide = torch.zeros((n, 3, 128), dtype=torch.bfloat16, device="cuda")
+    v_wide = torch.zeros((n, 3, 128), dtype=torch.bfloat16, device="cuda")
+    q, k, v = q_wide[:, 2:2 + hq], k_wide[:, 1:2], v_wide[:, 1:2]
+    q.copy_(to_dev(data["q"])); k.copy_(to_dev(data["k"])); v.copy_(to_dev(data["v"]))
+    out = torch.full((n, hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((hq, n), float("nan"), dtype=torch.float32, device="cuda")
+    binding.stem_token_attention(q, k, v, torch.from_numpy(idx_ref).cuda(), torch.from_numpy(cnt_ref).cuda(), out, lse)
+    st, detail = binding.stem_token_check_status()
+    assert st == 0, detail
+    ei, ec = so.expand_group_lists(idx_ref, cnt_ref, hq // hkv)
+    O_ref, lse_ref = so.attention(data["q"], data["k"], data["v"], data["cu_seqlens"], 1, ei, ec)
+    check_attention(from_dev_bf16(out), O_ref, label="hand-made token lists, 16 heads per kv head")
+    empty = cnt_ref[0] == 0
+    assert empty.any()
+    assert (from_dev_bf16(out)[empty] == 0).all()
+    got_lse = lse.cpu().numpy()
+    assert np.isneginf(got_lse[:, empty]).all() and np.isneginf(lse_ref[:, empty]).all()
+    assert np.abs(got_lse[:, ~empty] - lse_ref[:, ~empty]).max() < 1e-3
+
+
 def test_token_level_argument_errors():
     with pytest.raises(binding.StemError):
         binding.stem_token_budget(100, 10, (11, 10))
