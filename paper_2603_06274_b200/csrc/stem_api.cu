@@ -583,6 +583,7 @@ int stem_token_attention(const void* Q, const void* K, const void* V, int32_t n_
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(O)) return STEM_ERR_INVALID_ARG;
   if (n_tokens < 1 || num_q_heads < 1 || num_kv_heads < 1 || num_kv_heads > 65535 || k_max < 1) return STEM_ERR_INVALID_ARG;
   if (num_q_heads % num_kv_heads != 0 || num_q_heads / num_kv_heads > token_attn_max_group()) return STEM_ERR_UNSUPPORTED;
+  if ((int64_t)n_tokens * num_kv_heads > 0x7fffffffLL) return STEM_ERR_UNSUPPORTED;  // work items are counted in 32 bits
   if (q_stride_tok % 8 || q_stride_head % 8 || kv_stride_tok % 8 || kv_stride_head % 8) return STEM_ERR_INVALID_ARG;
   if (q_stride_head < kHeadDim || kv_stride_head < kHeadDim) return STEM_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.f)) return STEM_ERR_INVALID_ARG;
