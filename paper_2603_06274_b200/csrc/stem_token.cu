@@ -5,8 +5,9 @@
 // group share the selection), and attends over exactly those tokens.  This file holds the selection:
 //
 //   token_select_kernel   one CTA per (list head, query token): exact top-k of the row's candidates by
-//                         (score descending, token id ascending) with a four-pass radix selection on
-//                         order-preserving keys through shared-memory histograms; the forced tokens (the first
+//                         (score descending, token id ascending) with a radix selection, a byte per pass, on
+//                         order-preserving keys through shared-memory histograms (it stops as soon as the bin that
+//                         holds the rank is taken whole); the forced tokens (the first
 //                         `stem` and the last `local`, the token itself included) are kept outside the
 //                         ranking; the list comes out ascending.  The row's keys are converted once into
 //                         shared memory (rows of up to 51 200 tokens; longer rows are re-read from the L2).
@@ -47,7 +48,7 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
   extern __shared__ uint32_t s_keys[];
   __shared__ int hist[kSelThreads / 32][256];  // one histogram per warp: fewer colliding atomics
   __shared__ uint32_t s_prefix;
-  __shared__ int s_need;
+  __shared__ int s_need, s_whole;
   const int t = N - 1 - (int)blockIdx.x;  // long rows first
   const int lh = blockIdx.y;
   const int warp = threadIdx.x >> 5;
@@ -67,10 +68,12 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
     __syncthreads();
   }
   // ---- the need-th largest key: most significant byte first, a histogram per byte
-  uint32_t prefix = 0u;  // the bytes decided so far (in the high bits)
-  int k = need;          // rank wanted among the keys that match the prefix
+  uint32_t prefix = 0u;   // the bytes decided so far (in the high bits)
+  uint32_t decided = 0u;  // their bit mask
+  int k = need;           // rank wanted among the keys that match the prefix
+  bool whole = false;     // the bin that holds the rank is taken whole: the remaining bytes need no pass
   if (ranked) {
-    for (int pass = 0; pass < 4; ++pass) {
+    for (int pass = 0; pass < 4 && !whole; ++pass) {
       const int shift = 24 - 8 * pass;
       const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
 #pragma unroll
@@ -111,15 +114,19 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
           }
           s_prefix = prefix | ((uint32_t)b << shift);
           s_need = k - acc;
+          s_whole = hist[0][b] == k - acc;
         }
       }
       __syncthreads();
       prefix = s_prefix;
       k = s_need;
+      whole = s_whole != 0;
+      decided |= 0xffu << shift;
       __syncthreads();
     }
   }
-  // keys above `prefix` are taken, of the keys equal to it the first k by token id
+  // keys whose decided bytes are above `prefix` are taken; of those equal to it all (whole) or the first k by token id
+  const int k_eq = whole ? 0x7fffffff : k;
 
   // ---- emission in ascending token order: stem tokens, selected candidates, local tokens
   for (int j = threadIdx.x; j < n_stem; j += kSelThreads) out[j] = j;
@@ -138,8 +145,8 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
     for (int c0 = s_lo; c0 < s_hi; c0 += 32) {
       const int c = c0 + lane;
       const uint32_t key = c < s_hi ? key_at(c) : 0u;
-      n_gt += __popc(__ballot_sync(0xffffffffu, c < s_hi && key > prefix));
-      n_eq += __popc(__ballot_sync(0xffffffffu, c < s_hi && key == prefix));
+      n_gt += __popc(__ballot_sync(0xffffffffu, c < s_hi && (key & decided) > prefix));
+      n_eq += __popc(__ballot_sync(0xffffffffu, c < s_hi && (key & decided) == prefix));
     }
     __shared__ int seg_gt[kSelThreads / 32], seg_eq[kSelThreads / 32];
     if (lane == 0) { seg_gt[warp] = n_gt; seg_eq[warp] = n_eq; }
@@ -147,7 +154,7 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
     int eq_before = 0, pos = n_stem, all_sel = 0;
 #pragma unroll
     for (int w = 0; w < kSelThreads / 32; ++w) {
-      const int take = seg_gt[w] + min(max(k - eq_before_all(seg_eq, w), 0), seg_eq[w]);
+      const int take = seg_gt[w] + min(max(k_eq - eq_before_all(seg_eq, w), 0), seg_eq[w]);
       if (w < warp) { pos += take; eq_before += seg_eq[w]; }
       all_sel += take;
     }
@@ -155,10 +162,10 @@ __global__ void __launch_bounds__(kSelThreads) token_select_kernel(const float* 
     for (int c0 = s_lo; c0 < s_hi; c0 += 32) {
       const int c = c0 + lane;
       const uint32_t key = c < s_hi ? key_at(c) : 0u;
-      const bool gt = c < s_hi && key > prefix;
-      const bool eq = c < s_hi && key == prefix;
+      const bool gt = c < s_hi && (key & decided) > prefix;
+      const bool eq = c < s_hi && (key & decided) == prefix;
       const uint32_t eq_mask = __ballot_sync(0xffffffffu, eq);
-      const bool sel = gt || (eq && eq_before + __popc(eq_mask & below) < k);
+      const bool sel = gt || (eq && eq_before + __popc(eq_mask & below) < k_eq);
       const uint32_t sel_mask = __ballot_sync(0xffffffffu, sel);
       if (sel) out[pos + __popc(sel_mask & below)] = c;
       pos += __popc(sel_mask);
