@@ -114,6 +114,47 @@ def test_gather_attention_on_hand_made_lists_with_strided_tensors():
     assert np.abs(got_lse[:, ~empty] - lse_ref[:, ~empty]).max() < 1e-3
 
 
+@pytest.mark.parametrize("seed", [31, 32, 33, 34, 35, 36])
+def test_gather_attention_on_random_shapes_and_list_lengths(seed):
+    # item boundaries in every phase of the pipeline: lists of 0 .. 3 tiles in random order, any group size; the
+    # result must also be the same bits on a second run
+    r = np.random.default_rng(seed)
+    hkv = int(r.integers(1, 4))
+    g = int(r.choice([1, 2, 3, 4, 5, 8, 12, 16]))
+    hq = hkv * g
+    n = int(r.integers(130, 420))
+    w = wl.small(f"token_fuzz_{seed}", seqlens=(n,), hq=hq, hkv=hkv, block=64, permille=100, sink=bool(seed & 1), seed=seed)
+    data = wl.make_qkv(w)
+    k_max = int(r.integers(1, n + 1))
+    idx_ref = np.full((hkv, n, k_max), -1, np.int32)
+    cnt_ref = np.zeros((hkv, n), np.int32)
+    for h in range(hkv):
+        for t in range(n):
+            top = min(t + 1, k_max)
+            m = int(r.choice([0, 1, min(top, 127), min(top, 128), min(top, 129), top, int(r.integers(0, top + 1))]))
+            idx_ref[h, t, :m] = np.sort(r.choice(t + 1, size=m, replace=False))
+            cnt_ref[h, t] = m
+    q, k, v = to_dev(data["q"]), to_dev(data["k"]), to_dev(data["v"])
+    idx, cnt = torch.from_numpy(idx_ref).cuda(), torch.from_numpy(cnt_ref).cuda()
+    outs = []
+    for _ in range(2):
+        out = torch.full((n, hq, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((hq, n), float("nan"), dtype=torch.float32, device="cuda")
+        binding.stem_token_attention(q, k, v, idx, cnt, out, lse)
+        st, detail = binding.stem_token_check_status()
+        assert st == 0, detail
+        outs.append((out, lse))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+    assert torch.equal(outs[0][1].view(torch.int32), outs[1][1].view(torch.int32))
+    ei, ec = so.expand_group_lists(idx_ref, cnt_ref, g)
+    O_ref, lse_ref = so.attention(data["q"], data["k"], data["v"], data["cu_seqlens"], 1, ei, ec)
+    check_attention(from_dev_bf16(outs[0][0]), O_ref, label=f"random token lists, n={n}, {hq}/{hkv} heads, k_max={k_max}")
+    got = outs[0][1].cpu().numpy()
+    empty = np.repeat(cnt_ref == 0, g, axis=0)
+    assert np.isneginf(got[empty]).all()
+    assert np.abs(got[~empty] - lse_ref[~empty]).max() < 1e-3
+
+
 def test_token_level_argument_errors():
     with pytest.raises(binding.StemError):
         binding.stem_token_budget(100, 10, (11, 10))
