@@ -44,11 +44,13 @@ namespace {
 
 constexpr int kThreads = 384;
 constexpr int kTileM = 128;
-constexpr int kKvSlots = 5;
+constexpr int kKvSlotsMax = 5;                            // K / V ring: 5 slots, or 4 with a spare Q tile
+constexpr int kQBufsMax = 3;                             // Q tiles: one per slot, or three (a spare for the next item's tile)
 constexpr int kSlotBytes = 32 * 1024;
 constexpr int kQBytes = 32 * 1024;
 constexpr int kTmemCols = 512;
 constexpr int kCmdSlots = 4;
+constexpr int kSpareQMaxList = 256;                      // longest list (blocks) served with the spare Q tile
 constexpr int kOCol = 256;                               // O of slot X at kOCol + 128 X; S/P at 128 X
 constexpr uint64_t kWaitLimitNs = 400ull * 1000 * 1000;  // per wait
 constexpr float kRescaleThreshold = 8.0f;                // log2 units
@@ -64,14 +66,13 @@ enum Cmd : uint32_t { kCmdPv = 1u, kCmdQk = 2u, kCmdPvFirst = 4u, kCmdPvLast = 8
 
 struct Smem {
   // offsets from the 1024-aligned base
-  static constexpr int q = 0;                             // two Q tiles
-  static constexpr int kv = q + 2 * kQBytes;              // K / V ring
-  static constexpr int bars = kv + kKvSlots * kSlotBytes;
+  static constexpr int q = 0;                             // the Q tiles, then the K / V ring: 7 x 32 KB together
+  static constexpr int bars = q + 7 * kSlotBytes;
   static constexpr int kv_full = bars;
-  static constexpr int kv_empty = kv_full + 8 * kKvSlots;
-  static constexpr int q_full = kv_empty + 8 * kKvSlots;
-  static constexpr int q_empty = q_full + 16;
-  static constexpr int s_full = q_empty + 16;
+  static constexpr int kv_empty = kv_full + 8 * kKvSlotsMax;
+  static constexpr int q_full = kv_empty + 8 * kKvSlotsMax;
+  static constexpr int q_empty = q_full + 8 * kQBufsMax;
+  static constexpr int s_full = q_empty + 8 * kQBufsMax;
   static constexpr int p_ready = s_full + 16;
   static constexpr int p_early = p_ready + 16;            // all of P but its last 32 key columns stored
   static constexpr int o_full = p_early + 16;
@@ -86,6 +87,7 @@ struct Smem {
 };
 constexpr int kSmemBytes = Smem::total + 1024;  // slack for manual 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(kQBytes == kSlotBytes, "a Q tile and a ring slot trade places one for one");
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -349,7 +351,7 @@ struct ItemCursor {
   }
 };
 
-template <int BLK>
+template <int BLK, bool kSpareQ>
 __global__ void __launch_bounds__(kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const AttnArgs a) {
@@ -361,12 +363,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
   volatile int* abort_flag = (volatile int*)(smem_gen + Smem::abort_flag);
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem_gen + Smem::tmem_ptr);
   auto bar = [&](int off, int idx) { return smem_base + off + 8 * idx; };
+  // kSpareQ: three Q tiles (the next item's tile is loaded into a spare while the current items run) and a ring of
+  // four K / V slots, for lists of tens of blocks, where an item boundary that waits for Q costs two blocks' time;
+  // otherwise two Q tiles and a ring of five, for long lists (and the dense mode), where the deeper ring pays.
+  constexpr int kKvSlots = kSpareQ ? 4 : 5;
+  constexpr int kQBufs = kSpareQ ? 3 : 2;
+  constexpr int kKvOff = Smem::q + kQBufs * kQBytes;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kKvSlots; ++i) { mbar_init(bar(Smem::kv_full, i), 1); mbar_init(bar(Smem::kv_empty, i), 1); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kQBufs; ++i) {
       mbar_init(bar(Smem::q_full, i), 1);
       mbar_init(bar(Smem::q_empty, i), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(bar(Smem::s_full, i), 1);
       mbar_init(bar(Smem::p_ready, i), 4);   // one arrival per softmax warp
       mbar_init(bar(Smem::p_early, i), 4);   // likewise
@@ -584,7 +594,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       uint32_t kv_prod = 0;             // copies issued so far
       auto load = [&](const CUtensorMap* map, int kvh, int tok) -> bool {
         if (!__all_sync(0xffffffffu, mbar_wait(bar(Smem::kv_empty, ring), ring_par ^ 1, ctx, kBarKvEmpty))) return false;
-        const uint32_t dst = smem_base + Smem::kv + ring * kSlotBytes;
+        const uint32_t dst = smem_base + kKvOff + ring * kSlotBytes;
         if (elect_one()) {
           mbar_expect_tx(bar(Smem::kv_full, ring), kKvTileBytes);
           tma_load_3d(dst, map, bar(Smem::kv_full, ring), 0, kvh, tok);
@@ -617,9 +627,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       s0.pend = s1.pend = false;
       enter(s0); enter(s1);
       bool ok = true;
-      while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
+      // With the spare Q tile slot 1 starts half an item behind slot 0, so that the two slots' item boundaries (and
+      // their claims on the spare) do not fall together.  The scheduler skips the same visits.
+      const uint32_t delay1 = (kSpareQ && s0.has) ? (uint32_t)s0.cur.n / 2u : 0u;
+      for (uint32_t it = 0; ok && (s0.has || s1.has || s0.pend || s1.pend); ++it) {
         ok = visit(s0);
-        if (ok) ok = visit(s1);
+        if (ok && (!kSpareQ || it >= delay1)) ok = visit(s1);
       }
       if (!ok && lane == 0) {
         // aborting: give copies already in flight a bounded time to land before the CTA exits
@@ -632,44 +645,96 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     } else if (warp == 10) {
       // ============================== Q producer ==============================
       Ctx ctx{abort_flag, a.status, kRoleQProducer};
-      ItemCursor c0, c1;
-      c0.init(0); c1.init(1);
-      bool has0 = c0.next(a), has1 = c1.next(a);
-      uint32_t ord0 = 0, ord1 = 0;
-      // Loads the slot's next Q tile as soon as the last Q K^T of its previous item has read the buffer.
-      auto try_load = [&](ItemCursor& cur, bool& has, uint32_t& ord, const int X) -> bool {
-        if (!has || !uni((int)mbar_test(bar(Smem::q_empty, X), (ord & 1) ^ 1))) return false;
-        const int q_tok0 = uni(a.rows.row_tok0[cur.R]);
-        const uint32_t dst = smem_base + Smem::q + X * kQBytes;
-        if (elect_one()) {
-          mbar_expect_tx(bar(Smem::q_full, X), kQBytes);
-          tma_load_3d(dst, &map_q, bar(Smem::q_full, X), 0, cur.h, q_tok0);
-          tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, X), 64, cur.h, q_tok0);
+      if constexpr (kSpareQ) {
+        // The two slots advance one block per scheduler iteration, so the iteration at which a slot's item ends is the
+        // running sum of its list lengths: the slot with the smaller sum finishes first (slot 0 on a tie) and gets the
+        // next tile, loaded into the spare buffer long before it is wanted; the buffer the slot leaves becomes the
+        // spare once the last Q K^T of its item has read it.  The scheduler rotates the buffers by the same rule.
+        ItemCursor c0, c1;
+        c0.init(0); c1.init(1);
+        bool has0 = c0.next(a), has1 = c1.next(a);
+        uint32_t q_used = 0u, q_odd = 0u;  // per buffer (bit b): a tile was loaded; an odd number of tiles was loaded
+        bool ok = true;
+        auto load_into = [&](const ItemCursor& cur, const int b) -> bool {
+          if (((q_used >> b) & 1u) &&
+              !__all_sync(0xffffffffu, mbar_wait(bar(Smem::q_empty, b), ((q_odd >> b) & 1u) ^ 1u, ctx, kBarQEmpty)))
+            return false;
+          const int q_tok0 = uni(a.rows.row_tok0[cur.R]);
+          const uint32_t dst = smem_base + Smem::q + b * kQBytes;
+          if (elect_one()) {
+            mbar_expect_tx(bar(Smem::q_full, b), kQBytes);
+            tma_load_3d(dst, &map_q, bar(Smem::q_full, b), 0, cur.h, q_tok0);
+            tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, b), 64, cur.h, q_tok0);
+          }
+          __syncwarp();
+          q_used |= 1u << b;
+          q_odd ^= 1u << b;
+          return true;
+        };
+        uint32_t end0 = 0, end1 = 0;  // scheduler iteration at which the slot's latest loaded item ends
+        int buf0 = 0, buf1 = 1, spare = 2;
+        const uint32_t delay1 = has0 ? (uint32_t)c0.n / 2u : 0u;  // slot 1 starts this many iterations late
+        if (has0) { ok = load_into(c0, buf0); end0 = (uint32_t)c0.n; has0 = c0.next(a); }
+        if (ok && has1) { ok = load_into(c1, buf1); end1 = delay1 + (uint32_t)c1.n; has1 = c1.next(a); }
+        while (ok && (has0 || has1)) {
+          if (has0 && (!has1 || end0 <= end1)) {
+            ok = load_into(c0, spare);
+            const int old = buf0; buf0 = spare; spare = old;
+            end0 += (uint32_t)c0.n;
+            has0 = c0.next(a);
+          } else {
+            ok = load_into(c1, spare);
+            const int old = buf1; buf1 = spare; spare = old;
+            end1 += (uint32_t)c1.n;
+            has1 = c1.next(a);
+          }
         }
-        __syncwarp();
-        ++ord;
-        has = cur.next(a);
-        return true;
-      };
-      bool ok = true;
-      uint64_t t0 = globaltimer();
-      uint32_t spin = 0;
-      while (ok && (has0 || has1)) {
-        const bool p0 = try_load(c0, has0, ord0, 0);
-        const bool p1 = try_load(c1, has1, ord1, 1);
-        if (p0 || p1) { t0 = globaltimer(); spin = 0; continue; }
-        __nanosleep(400);  // a Q tile is wanted once per item: poll slowly, the issue slots belong to the softmax warps
-        if ((++spin & 31u) == 0u) {
-          bool stop = *abort_flag != 0;
-          if (!stop && globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); stop = true; }
-          if (__any_sync(0xffffffffu, stop)) ok = false;
+        if (!ok && lane == 0) {
+          // aborting: bounded wait for Q copies that may still be in flight
+          const uint64_t t1 = globaltimer();
+          for (int b = 0; b < kQBufs; ++b)
+            while (((q_used >> b) & 1u) && !mbar_try(bar(Smem::q_full, b), ((q_odd >> b) & 1u) ^ 1u) && globaltimer() - t1 < 4000000ull) {}
         }
-      }
-      if (!ok && lane == 0) {
-        // aborting: bounded wait for a Q copy that may still be in flight
-        const uint64_t t1 = globaltimer();
-        while (ord0 > 0 && !mbar_try(bar(Smem::q_full, 0), (ord0 - 1) & 1) && globaltimer() - t1 < 2000000ull) {}
-        while (ord1 > 0 && !mbar_try(bar(Smem::q_full, 1), (ord1 - 1) & 1) && globaltimer() - t1 < 4000000ull) {}
+      } else {
+        ItemCursor c0, c1;
+        c0.init(0); c1.init(1);
+        bool has0 = c0.next(a), has1 = c1.next(a);
+        uint32_t ord0 = 0, ord1 = 0;
+        // Loads the slot's next Q tile as soon as the last Q K^T of its previous item has read the buffer.
+        auto try_load = [&](ItemCursor& cur, bool& has, uint32_t& ord, const int X) -> bool {
+          if (!has || !uni((int)mbar_test(bar(Smem::q_empty, X), (ord & 1) ^ 1))) return false;
+          const int q_tok0 = uni(a.rows.row_tok0[cur.R]);
+          const uint32_t dst = smem_base + Smem::q + X * kQBytes;
+          if (elect_one()) {
+            mbar_expect_tx(bar(Smem::q_full, X), kQBytes);
+            tma_load_3d(dst, &map_q, bar(Smem::q_full, X), 0, cur.h, q_tok0);
+            tma_load_3d(dst + kTileM * 128, &map_q, bar(Smem::q_full, X), 64, cur.h, q_tok0);
+          }
+          __syncwarp();
+          ++ord;
+          has = cur.next(a);
+          return true;
+        };
+        bool ok = true;
+        uint64_t t0 = globaltimer();
+        uint32_t spin = 0;
+        while (ok && (has0 || has1)) {
+          const bool p0 = try_load(c0, has0, ord0, 0);
+          const bool p1 = try_load(c1, has1, ord1, 1);
+          if (p0 || p1) { t0 = globaltimer(); spin = 0; continue; }
+          __nanosleep(400);  // a Q tile is wanted once per item: poll slowly, the issue slots belong to the softmax warps
+          if ((++spin & 31u) == 0u) {
+            bool stop = *abort_flag != 0;
+            if (!stop && globaltimer() - t0 > kWaitLimitNs) { raise_abort(ctx, kBarQEmpty); stop = true; }
+            if (__any_sync(0xffffffffu, stop)) ok = false;
+          }
+        }
+        if (!ok && lane == 0) {
+          // aborting: bounded wait for a Q copy that may still be in flight
+          const uint64_t t1 = globaltimer();
+          while (ord0 > 0 && !mbar_try(bar(Smem::q_full, 0), (ord0 - 1) & 1) && globaltimer() - t1 < 2000000ull) {}
+          while (ord1 > 0 && !mbar_try(bar(Smem::q_full, 1), (ord1 - 1) & 1) && globaltimer() - t1 < 4000000ull) {}
+        }
       }
     } else if (warp == 9) {
       // ============================== MMA scheduler ==============================
@@ -686,8 +751,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         bool has, pend, pend_first, pend_last;
         int e;
         uint32_t p_par, q_par, o_par;  // phase parities of p_ready, q_full, o_full / o_free
+        int qbuf;                      // Q buffer of the slot's current item
       };
       uint32_t ring = 0, ring_par = 0;  // next K / V ring slot to consume and its phase
+      int q_spare = 2;      // kSpareQ: the buffer that receives the next item's tile, and per buffer (bit b) whether an
+      uint32_t q_odd = 3u;  // odd number of items was assigned to it so far - the Q producer's rule, step for step
       // One visit.  Every barrier the visit depends on is probed up front in one go (independent
       // shared-memory operations in flight together); only a failed probe falls back to the bounded waits.
       auto visit = [&](MmaSlot& s, const int X) -> bool {
@@ -699,13 +767,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const bool last = do_qk && s.e == s.cur.n - 1;
         const uint32_t all_done =
             mbar_try4(bar(Smem::kv_full, slot_v), par_v, do_pv, bar(Smem::o_free, X), s.o_par ^ 1, need_o,
-                      bar(Smem::kv_full, slot_k), par_k, do_qk, bar(Smem::q_full, X), s.q_par, need_q);
+                      bar(Smem::kv_full, slot_k), par_k, do_qk, bar(Smem::q_full, s.qbuf), s.q_par, need_q);
         if (!__all_sync(0xffffffffu, all_done != 0)) {
           bool ok = true;
           if (do_pv) ok = mbar_wait(bar(Smem::kv_full, slot_v), par_v, ctx, kBarKvFull);
           if (ok && need_o) ok = mbar_wait(bar(Smem::o_free, X), s.o_par ^ 1, ctx, kBarOFree);
           if (ok && do_qk) ok = mbar_wait(bar(Smem::kv_full, slot_k), par_k, ctx, kBarKvFull);
-          if (ok && need_q) ok = mbar_wait(bar(Smem::q_full, X), s.q_par, ctx, kBarQFull);
+          if (ok && need_q) ok = mbar_wait(bar(Smem::q_full, s.qbuf), s.q_par, ctx, kBarQFull);
           if (!__all_sync(0xffffffffu, ok)) return false;
         }
         // everything the visit needs is in place: hand it to the issuing warp
@@ -713,7 +781,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (lane == 0) {
           cmd_word[ci] = (do_pv ? kCmdPv : 0u) | (do_qk ? kCmdQk : 0u) | (s.pend_first ? kCmdPvFirst : 0u) |
                          (s.pend_last ? kCmdPvLast : 0u) | (last ? kCmdQkLast : 0u) | (X ? kCmdSlot1 : 0u) |
-                         (s.p_par ? kCmdPPar : 0u) | (slot_v << 8) | (slot_k << 12);
+                         (s.p_par ? kCmdPPar : 0u) | (slot_v << 8) | (slot_k << 12) | ((uint32_t)s.qbuf << 16);
           mbar_arrive(bar(Smem::cmd_full, ci));  // release: the word and everything observed above
         }
         __syncwarp();
@@ -730,9 +798,19 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
           s.pend_first = s.e == 0;
           s.pend_last = last;
           if (last) {
-            s.q_par ^= 1;
             s.has = s.cur.next(a);
             s.e = 0;
+            if constexpr (kSpareQ) {
+              if (s.has) {  // the next item's tile is (or will be) in the spare buffer; this item's buffer becomes the spare
+                const int old = s.qbuf;
+                s.qbuf = q_spare;
+                q_spare = old;
+                s.q_par = (q_odd >> s.qbuf) & 1u;
+                q_odd ^= 1u << s.qbuf;
+              }
+            } else {
+              s.q_par ^= 1;
+            }
           } else {
             ++s.e;
           }
@@ -745,10 +823,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       s0.pend = s1.pend = s0.pend_first = s1.pend_first = s0.pend_last = s1.pend_last = false;
       s0.e = s1.e = 0;
       s0.p_par = s1.p_par = s0.q_par = s1.q_par = s0.o_par = s1.o_par = 0;
+      s0.qbuf = 0; s1.qbuf = 1;
       bool ok = true;
-      while (ok && (s0.has || s1.has || s0.pend || s1.pend)) {
+      const uint32_t delay1 = (kSpareQ && s0.has) ? (uint32_t)s0.cur.n / 2u : 0u;  // as in the K / V producer
+      for (uint32_t it = 0; ok && (s0.has || s1.has || s0.pend || s1.pend); ++it) {
         ok = visit(s0, 0);
-        if (ok) ok = visit(s1, 1);
+        if (ok && (!kSpareQ || it >= delay1)) ok = visit(s1, 1);
       }
       // tell the issuing warp that nothing follows (also when aborting: its own waits are bounded too)
       if (__all_sync(0xffffffffu, mbar_wait(bar(Smem::cmd_empty, ci), cpar ^ 1, ctx, kBarCmdEmpty)) && lane == 0) {
@@ -777,7 +857,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t s_tmem = tmem_base + X * 128;
         const uint32_t o_tmem = tmem_base + kOCol + X * 128;
         constexpr int kEarlySteps = (BLK / 32 - 1) * 2;  // 16-key steps of P V covered by p_early
-        const uint32_t v_addr = smem_base + Smem::kv + slot_v * kSlotBytes;
+        const uint32_t v_addr = smem_base + kKvOff + slot_v * kSlotBytes;
         const uint32_t p_par = (cmd & kCmdPPar) ? 1u : 0u;
         if (cmd & kCmdPv) {
           // The one condition the scheduler leaves open: the slot's softmax warps have stored P.
@@ -813,8 +893,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             if (cmd & kCmdPvLast) tc_commit(bar(Smem::o_full, X));
           }
           if (cmd & kCmdQk) {
-            const uint32_t q_addr = smem_base + Smem::q + X * kQBytes;
-            const uint32_t k_addr = smem_base + Smem::kv + slot_k * kSlotBytes;
+            const uint32_t qb = (cmd >> 16) & 3u;
+            const uint32_t q_addr = smem_base + Smem::q + qb * kQBytes;
+            const uint32_t k_addr = smem_base + kKvOff + slot_k * kSlotBytes;
             uint64_t da = smem_desc(q_addr, 16, 1024);
             uint64_t db = smem_desc(k_addr, 16, 1024);
             uint32_t acc = 0u;
@@ -828,7 +909,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             tc_commit(bar(Smem::kv_empty, slot_k));
             tc_commit(bar(Smem::s_full, X));
-            if (cmd & kCmdQkLast) tc_commit(bar(Smem::q_empty, X));
+            if (cmd & kCmdQkLast) tc_commit(bar(Smem::q_empty, qb));
           }
         }
         __syncwarp();
@@ -892,17 +973,24 @@ cudaError_t launch_sparse_attention(const Plan& p, const void* Q, const void* K,
   static bool attr_set[64] = {};
   const int dev_slot = p.device & 63;
   if (!attr_set[dev_slot]) {
-    e = cudaFuncSetAttribute(sparse_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(sparse_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(sparse_attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sparse_attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sparse_attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(sparse_attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set[dev_slot] = true;
   }
   const int grid = std::min(p.n_items, p.sm_count);
-  if (B == 128)
-    sparse_attn_kernel<128><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
-  else
-    sparse_attn_kernel<64><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
+  // Lists of up to a few hundred blocks: the spare Q tile (an item boundary then costs no wait for Q); the dense mode
+  // and longer lists: the deeper K / V ring.
+  const bool spare_q = sel_idx != nullptr && p.k_max <= kSpareQMaxList;
+  if (B == 128) {
+    if (spare_q) sparse_attn_kernel<128, true><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
+    else sparse_attn_kernel<128, false><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
+  } else {
+    if (spare_q) sparse_attn_kernel<64, true><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
+    else sparse_attn_kernel<64, false><<<grid, kThreads, kSmemBytes, s>>>(mq, mk, mv, a);
+  }
   return cudaGetLastError();
 }
 

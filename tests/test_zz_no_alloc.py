@@ -6,6 +6,8 @@ whose pool already owns the GPU, or in callbacks where the host framework forbid
 calls.  For them the library keeps the pooled tensors of the scoring stage in a fixed array of
 its own.  This file is collected last on purpose, so that a failure here cannot hide the result
 of any other test in a run that stops at the first failure."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -16,6 +18,11 @@ from paper_2603_06274_b200.binding import StemPlan
 from tests._util import oracle_params, to_dev
 
 pytestmark = pytest.mark.gpu
+
+
+def _allocation_requests() -> int:
+    """How many blocks torch's CUDA allocator has handed out since the process started."""
+    return int(torch.cuda.memory_stats().get("allocation.all.allocated", 0))
 
 
 def _metric_triple(w):
@@ -29,13 +36,17 @@ def _metric_triple(w):
     got = torch.full((w.num_q_heads, n), float("nan"), dtype=torch.float32, device="cuda")
     binding.stem_score(plan, q, k, v, want)          # existing entry point, caller workspace
     torch.cuda.synchronize()
-    # the call under test must not request device memory: neither through torch's allocator nor from the driver
-    torch_before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved())
+    # the call under test must not request device memory: neither through torch's allocator nor from the driver.
+    # (Counted as allocation requests, not as bytes in use: tensors left behind by earlier tests may be released by
+    # Python's collector at any moment, which lowers the bytes in use without anybody having asked for memory.)
+    gc.collect()
+    torch.cuda.synchronize()
+    torch_before = (_allocation_requests(), torch.cuda.memory_reserved())
     free_before, _ = torch.cuda.mem_get_info()
     binding.stem_score_static(plan, q, k, v, got)    # same stage, library-owned scratch
     torch.cuda.synchronize()
     free_after, _ = torch.cuda.mem_get_info()
-    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == torch_before
+    assert (_allocation_requests(), torch.cuda.memory_reserved()) == torch_before
     assert free_after == free_before, "the driver's free-memory count changed across the call"
     assert binding.stem_check_status(plan, static_scratch=True)[0] == binding.STEM_OK
     ref, *_ = so.score(data["q"], data["k"], data["v"], data["cu_seqlens"], oracle_params(w))
