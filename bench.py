@@ -34,8 +34,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # DRAM traffic of one sparse-attention launch (ncu: dram__bytes_read.sum + dram__bytes_write.sum),
 # captured on the workload itself; a workload without a capture reports null.
-NCU_ATTN_DRAM_BYTES_PER_LAUNCH = {"cfg3_llama3_8b_128k": 1680473088 + 1047045120,
-                                  "cfg2_llama3_8b_32k": 404025344 + 240033536}
+NCU_ATTN_DRAM_BYTES_PER_LAUNCH = {"cfg3_llama3_8b_128k": 1631425792 + 1041603328,
+                                  "cfg2_llama3_8b_32k": 405131776 + 236100096}
 
 
 def load_peaks():

@@ -23,6 +23,10 @@
 // producer walks the same visit sequence, so one shared ring serves both slots in order.  A slot's
 // items follow each other without a gap: Q K^T of the next item's first block is issued right
 // behind P V of the previous item's last block while the slot's softmax warps drain O.
+// For that the next item's Q tile has to be there already: with lists of tens of blocks (kSpareQ) the
+// seven 32 KB tiles of shared memory are three Q tiles and a ring of four, the next tile is loaded into
+// the spare one while both current items run, and slot 1 starts half an item late so that the slots'
+// boundaries alternate; otherwise (dense mode, very long lists) two Q tiles and a ring of five.
 // Registers are re-balanced with setmaxnreg: the kernel must not spill, because with 227 KB of
 // shared memory in use almost no L1 is left for local memory.
 // Every mbarrier wait is bounded in time; a wait that gives up raises a CTA-wide abort flag,
